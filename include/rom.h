@@ -1,0 +1,141 @@
+/* rom.h — C ABI of the B200 (sm_100a) forward pass of one Routing-Mamba (RoM) layer.
+ *
+ * Paper notation (Sections 3.1 and 4.2): X in R^{L x D_m} per sequence, D_e = d_inner,
+ * D_s = d_state, k = d_conv, d_r = dt_rank, N experts = E, top-K.  T = B*L tokens in (b,t) order,
+ * "assignment" a = t*K + k is slot k of token t.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless marked "host".  The caller owns every buffer; the
+ *     library allocates no device memory and keeps no state on the device between calls.
+ *   - All tensors are dense, row-major, channels-last; device pointers must be 16-byte aligned.
+ *   - "dtype" tensors are stored as ROM_F32 (float) or ROM_BF16 (bfloat16) as rom_config.dtype says.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream);
+ *     they neither synchronise the host nor copy device memory to the host.
+ *   - Return value: a rom_status (0 = ok, negative = error).  Argument errors are found on the host
+ *     before anything is launched.  Device-side problems (a bounded wait that expired) are latched
+ *     in a status word at the head of the workspace and read with rom_get_status.
+ *   - Outputs are fully overwritten; inputs are never written; workspace contents are scratch.
+ *     Calls that use distinct workspaces and outputs are independent.
+ */
+#ifndef ROM_H_
+#define ROM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ROM_API __attribute__((visibility("default")))
+#else
+#define ROM_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { ROM_F32 = 0, ROM_BF16 = 1 } rom_dtype;
+
+typedef enum {
+  ROM_OK = 0,
+  ROM_ERR_INVALID_ARG = -1,    /* NULL required pointer, bad size, misaligned pointer            */
+  ROM_ERR_UNSUPPORTED = -2,    /* a legal problem this build does not cover (e.g. d_state != 16)   */
+  ROM_ERR_WORKSPACE = -3,      /* ws_bytes smaller than rom_workspace_size                        */
+  ROM_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (launch, tensor-map encode)   */
+  ROM_ERR_ARCH = -5,           /* the current device is not sm_100                                */
+  ROM_ERR_DEVICE_TIMEOUT = -6  /* a bounded device-side wait expired (reported by rom_get_status) */
+} rom_status;
+
+typedef struct {
+  int32_t B, L;               /* sequences, tokens per sequence                                   */
+  int32_t d_model, d_inner;   /* D_m, D_e : multiples of 64                                       */
+  int32_t d_state;            /* D_s : 16                                                         */
+  int32_t d_conv;             /* k : 2, 3 or 4                                                    */
+  int32_t dt_rank;            /* d_r : multiple of 16 (bf16) / of 4 (f32)                          */
+  int32_t E, K;               /* experts (1..64), top-K (1..min(E,8))                             */
+  int32_t dtype;              /* rom_dtype                                                        */
+  int32_t gate_mode;          /* 0: R_i = P_i * 1[i in TopK] (Section 4.2, routing equation);
+                                 1: P_i renormalised over the selected K (the sentence above it)   */
+  int32_t disc_mode;          /* 0: zero-order hold B-bar (Section 3.1); 1: B-bar = Delta * B      */
+  int32_t flags;              /* ROM_FLAG_* bits                                                  */
+  int32_t reserved;           /* must be 0                                                        */
+} rom_config;
+
+#define ROM_FLAG_SIMT_GEMM 1  /* run every projection on the plain fp32-FMA kernels (bisecting aid;
+                                 always the case for ROM_F32) instead of the tcgen05 tensor path   */
+
+typedef struct {                /* all read-only device pointers                                   */
+  const void  *W_r;             /* [E, d_model]              dtype  router, W_r of Section 4.2 transposed */
+  const float *b_r;             /* [E] or NULL               router bias (not in the paper)        */
+  const void  *W_inz;           /* [E, 2*d_inner, d_model]   dtype  rows [0,D_e): Conv Proj W_in,i^T,
+                                                                    rows [D_e,2D_e): Gate Proj W_g,i^T */
+  const void  *w_conv;          /* [d_conv, d_inner]         dtype  tap d_conv-1 = current token   */
+  const float *b_conv;          /* [d_inner] or NULL                                              */
+  const void  *W_x;             /* [dt_rank+2*d_state, d_inner] dtype  rows delta | B | C (shared) */
+  const void  *W_dt;            /* [d_inner, dt_rank]        dtype  (shared)                       */
+  const float *b_dt;            /* [d_inner] or NULL                                              */
+  const float *A;               /* [d_inner, d_state]        fp32, strictly negative              */
+  const float *D;               /* [d_inner] or NULL         skip (not in the paper's equations)   */
+  const void  *W_out;           /* [E, d_model, d_inner]     dtype  W_out,i^T                      */
+} rom_weights;
+
+/* Bytes of workspace rom_layer_forward / rom_route / rom_scan need for this config (host out).   */
+ROM_API int rom_workspace_size(const rom_config *cfg, size_t *bytes);
+
+/* Router + top-K + dropless permutation (Section 4.2 routing equation; Section 5.1: no capacity
+ * factor, no token dropping).
+ *   logit[t,e] = b_r[e] + sum_d x[t,d] W_r[e,d], accumulated in fp64 in ascending d;
+ *   P = softmax over all E; the K largest logits are selected, ties to the lowest expert id,
+ *   slot k = k-th largest; gates per gate_mode.
+ *   counts[e] = assignments of expert e; offsets = exclusive prefix sum (offsets[E] = T*K);
+ *   inside an expert's segment assignments keep ascending a = t*K+k:
+ *   perm[r] = a, inv_perm[a] = r.
+ * Outputs: topk_idx[T,K] i32, gates[T,K] f32, counts[E], offsets[E+1], perm[T*K], inv_perm[T*K] i32.
+ * Uses cfg->B, L, d_model, E, K, dtype, gate_mode.  Any output pointer may be NULL (not produced). */
+ROM_API int rom_route(const rom_config *cfg, const void *x, const void *W_r, const float *b_r,
+              int32_t *topk_idx, float *gates, int32_t *counts, int32_t *offsets,
+              int32_t *perm, int32_t *inv_perm, void *ws, size_t ws_bytes, void *stream);
+
+/* Selective scan (Section 3.1, linear recurrence h_t = A-bar h_{t-1} + B-bar U_t, Y_t = C h_t) with
+ * A-bar = exp(Delta A), B-bar per disc_mode, optional skip D*U and optional gate y *= SiLU(z)
+ * (output equation of Section 3.1).  State and arithmetic are fp32.
+ *   u, z, y : [B, L, d_inner] dtype;  delta : [B, L, d_inner] fp32;  A : [d_inner, d_state] fp32;
+ *   Bm, Cm : [B, L, d_state] fp32;  D : [d_inner] or NULL;  z NULL = no gate;
+ *   h0 : [B, d_inner, d_state] fp32 or NULL (zeros);  h_last : same shape or NULL (not produced).
+ * Uses cfg->B, L, d_inner, d_state, dtype, disc_mode.                                             */
+ROM_API int rom_scan(const rom_config *cfg, const void *u, const float *delta, const float *A,
+             const float *Bm, const float *Cm, const float *D, const void *z, const float *h0,
+             void *y, float *h_last, void *ws, size_t ws_bytes, void *stream);
+
+/* Forward pass of one RoM layer (Section 4.2 equations for G, H_t, O_t, E_i with the shared
+ * Conv1D / x Proj / dt Proj / A / D of Section 4.3):
+ *   route -> gather tokens by expert -> per-expert [Conv Proj | Gate Proj] -> un-permute, sum over
+ *   the selected experts (indicator only) -> causal depthwise conv + SiLU -> x Proj, dt Proj +
+ *   softplus -> selective scan -> * SiLU(gate) -> re-permute with the same routing -> per-expert
+ *   Out Proj -> gate-weighted sum over the selected experts.
+ *   x, out : [B, L, d_model] dtype.  topk_idx_out [T,K] i32, gates_out [T,K] f32, counts_out [E] i32
+ *   may each be NULL.                                                                             */
+ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const void *x, void *out,
+                      int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
+                      void *ws, size_t ws_bytes, void *stream);
+
+/* Locate a named intermediate of the last rom_layer_forward inside the workspace (host-only
+ * arithmetic; for tests and debugging).  Names: "U" [T,D_e] dtype, "delta_r" [T,d_r] dtype,
+ * "Bm","Cm" [T,D_s] f32, "Delta" [T,D_e] f32, "row_of_assign" [T*K] i32 (padded row of each
+ * assignment), "XZp" [rows,2*D_e] dtype, "Ygp" [rows,D_e] dtype, "pad_offsets" [E+1] i32.
+ * Returns ROM_ERR_INVALID_ARG for an unknown name.                                                */
+ROM_API int rom_workspace_find(const rom_config *cfg, const char *name, size_t *offset, size_t *bytes);
+
+/* Read and clear the device status word of a workspace.  `host_code` (host out) receives ROM_OK or
+ * ROM_ERR_DEVICE_TIMEOUT.  This call synchronises `stream`.                                       */
+ROM_API int rom_get_status(void *ws, void *stream, int32_t *host_code);
+
+/* Static string for a rom_status value.                                                           */
+ROM_API const char *rom_status_string(int code);
+
+/* Number of kernels the last call of rom_layer_forward launched on this host thread (host-only). */
+ROM_API int rom_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROM_H_ */

@@ -1,0 +1,158 @@
+"""Thin ctypes binding of the C ABI declared in include/rom.h: argument marshalling only.
+
+Every function takes torch tensors that already live where the ABI wants them (CUDA for data,
+none on the host except sizes) and forwards raw pointers.  Nothing here computes anything; when
+the compiled library is missing the import of `lib()` fails loudly -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librom_b200.so")
+
+ROM_F32, ROM_BF16 = 0, 1
+ROM_FLAG_SIMT_GEMM = 1
+ROM_OK = 0
+
+EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
+           "rom_get_status", "rom_status_string", "rom_last_launch_count")
+
+
+class RomConfig(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "L", "d_model", "d_inner", "d_state", "d_conv", "dt_rank", "E", "K", "dtype",
+                 "gate_mode", "disc_mode", "flags", "reserved")]
+
+
+class RomWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("W_r", "b_r", "W_inz", "w_conv", "b_conv", "W_x", "W_dt", "b_dt", "A", "D", "W_out")]
+
+
+class RomError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load librom_b200.so (built in-tree by paper_2506_18145_b200.build).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_18145_b200.build` "
+                              "(there is no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32p, szp = ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_size_t)
+        cfgp = ctypes.POINTER(RomConfig)
+        L.rom_workspace_size.argtypes = [cfgp, szp]
+        L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
+        L.rom_scan.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.rom_layer_forward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, i32p, vp, i32p, vp, ctypes.c_size_t, vp]
+        L.rom_workspace_find.argtypes = [cfgp, ctypes.c_char_p, szp, szp]
+        L.rom_get_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.rom_status_string.argtypes = [ctypes.c_int]
+        L.rom_status_string.restype = ctypes.c_char_p
+        L.rom_last_launch_count.argtypes = []
+        for name in EXPORTS:
+            if name != "rom_status_string":
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().rom_status_string(int(code)).decode()
+
+
+def make_config(B, L, d_model, d_inner, d_state, d_conv, dt_rank, E, K, dtype, gate_mode=0, disc_mode=0, flags=0) -> RomConfig:
+    dt = {"f32": ROM_F32, "bf16": ROM_BF16, torch.float32: ROM_F32, torch.bfloat16: ROM_BF16}[dtype]
+    return RomConfig(B, L, d_model, d_inner, d_state, d_conv, dt_rank, E, K, dt, gate_mode, disc_mode, flags, 0)
+
+
+def config_from_shape(shape, gate_mode=0, disc_mode=0, flags=0) -> RomConfig:
+    """shape: a synth.RomShape."""
+    return make_config(shape.B, shape.L, shape.d_model, shape.d_inner, shape.d_state, shape.d_conv, shape.dt_rank,
+                       shape.E, shape.K, shape.dtype, gate_mode, disc_mode, flags)
+
+
+def _ptr(t: Optional[torch.Tensor], cuda: bool = True) -> Optional[int]:
+    if t is None:
+        return None
+    if cuda and not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def workspace_size(cfg: RomConfig) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().rom_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_workspace_size")
+    return int(n.value)
+
+
+def workspace_find(cfg: RomConfig, name: str):
+    off, n = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    rc = lib().rom_workspace_find(ctypes.byref(cfg), name.encode(), ctypes.byref(off), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_workspace_find")
+    return int(off.value), int(n.value)
+
+
+def alloc_workspace(cfg: RomConfig, device="cuda") -> torch.Tensor:
+    return torch.empty(workspace_size(cfg), dtype=torch.uint8, device=device)
+
+
+def rom_route(cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm, ws, stream=None, check=True) -> int:
+    rc = lib().rom_route(ctypes.byref(cfg), _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(topk_idx), _ptr(gates), _ptr(counts),
+                         _ptr(offsets), _ptr(perm), _ptr(inv_perm), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_route")
+    return rc
+
+
+def rom_scan(cfg, u, delta, A, Bm, Cm, D, z, h0, y, h_last, ws=None, stream=None, check=True) -> int:
+    rc = lib().rom_scan(ctypes.byref(cfg), _ptr(u), _ptr(delta), _ptr(A), _ptr(Bm), _ptr(Cm), _ptr(D), _ptr(z), _ptr(h0),
+                        _ptr(y), _ptr(h_last), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_scan")
+    return rc
+
+
+def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> RomWeights:
+    return RomWeights(*[_ptr(w.get(n)) for n, _ in RomWeights._fields_])
+
+
+def rom_layer_forward(cfg, weights: RomWeights, x, out, topk_idx_out, gates_out, counts_out, ws, stream=None, check=True) -> int:
+    rc = lib().rom_layer_forward(ctypes.byref(cfg), ctypes.byref(weights), _ptr(x), _ptr(out), _ptr(topk_idx_out),
+                                 _ptr(gates_out), _ptr(counts_out), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_layer_forward")
+    return rc
+
+
+def rom_get_status(ws, stream=None) -> int:
+    code = ctypes.c_int32(0)
+    rc = lib().rom_get_status(_ptr(ws), _stream(stream), ctypes.byref(code))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_get_status")
+    return int(code.value)
+
+
+def last_launch_count() -> int:
+    return int(lib().rom_last_launch_count())

@@ -1,0 +1,249 @@
+// C ABI of the RoM layer forward: argument checks, workspace carving, launch sequence.
+#include <cstring>
+
+#include "rom_internal.cuh"
+
+namespace rom {
+
+thread_local int LaunchCounter::count = 0;
+
+WsLayout make_layout(const rom_config& c) {
+  WsLayout l{};
+  l.esz = c.dtype == ROM_BF16 ? 2 : 4;
+  l.T = (int64_t)c.B * c.L;
+  l.A = l.T * c.K;
+  // every expert segment is padded to a multiple of kTileM rows: at most kTileM-1 extra rows each
+  l.rows_max = (int64_t)align_up((size_t)l.A, kTileM) + (int64_t)c.E * kTileM;
+  l.max_m_tiles = l.rows_max / kTileM;
+  l.n_chunks = (l.T + kChunkTokens - 1) / kChunkTokens;
+  const int R = c.dt_rank, N = c.d_state;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  l.status = take(sizeof(int32_t) * kStatusInts);
+  l.counts = take(sizeof(int32_t) * c.E);
+  l.offsets = take(sizeof(int32_t) * (c.E + 1));
+  l.pad_offsets = take(sizeof(int32_t) * (c.E + 1));
+  l.num_m_tiles = take(sizeof(int32_t) * 4);
+  l.tile_expert = take(sizeof(int32_t) * l.max_m_tiles);
+  l.chunk_counts = take(sizeof(int32_t) * l.n_chunks * c.E);
+  l.topk_idx = take(sizeof(int32_t) * l.A);
+  l.gates = take(sizeof(float) * l.A);
+  l.perm = take(sizeof(int32_t) * l.A);
+  l.inv_perm = take(sizeof(int32_t) * l.A);
+  l.row_of_assign = take(sizeof(int32_t) * l.A);
+  l.assign_of_row = take(sizeof(int32_t) * l.rows_max);
+  l.x_perm = take(l.esz * (size_t)l.rows_max * c.d_model);
+  l.XZp = take(l.esz * (size_t)l.rows_max * 2 * c.d_inner);
+  l.U = take(l.esz * (size_t)l.T * c.d_inner);
+  l.delta_r = take(l.esz * (size_t)l.T * R);
+  l.Bm = take(sizeof(float) * (size_t)l.T * N);
+  l.Cm = take(sizeof(float) * (size_t)l.T * N);
+  l.Delta = take(sizeof(float) * (size_t)l.T * c.d_inner);
+  l.Ygp = take(l.esz * (size_t)l.rows_max * c.d_inner);
+  l.Op = take(l.esz * (size_t)l.rows_max * c.d_model);
+  l.total = o;
+  return l;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// which == 0: full layer; 1: route only; 2: scan only
+int check_config(const rom_config* c, int which) {
+  if (!c) return ROM_ERR_INVALID_ARG;
+  if (c->dtype != ROM_F32 && c->dtype != ROM_BF16) return ROM_ERR_INVALID_ARG;
+  if (c->B < 1 || c->L < 1) return ROM_ERR_INVALID_ARG;
+  if (c->reserved != 0 || (c->flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
+  if (which != 2) {
+    if (c->E < 1 || c->K < 1 || c->K > c->E) return ROM_ERR_INVALID_ARG;
+    if (c->E > kMaxE || c->K > kMaxK) return ROM_ERR_UNSUPPORTED;
+    if (c->gate_mode != 0 && c->gate_mode != 1) return ROM_ERR_INVALID_ARG;
+    if (c->d_model < 64 || c->d_model % 64 != 0) return ROM_ERR_INVALID_ARG;
+    if ((int64_t)c->B * c->L * c->K >= (int64_t)1 << 30) return ROM_ERR_UNSUPPORTED;
+  }
+  if (which != 1) {
+    if (c->d_inner < 64 || c->d_inner % 64 != 0) return ROM_ERR_INVALID_ARG;
+    if (c->d_state < 1) return ROM_ERR_INVALID_ARG;
+    if (c->d_state != 16) return ROM_ERR_UNSUPPORTED;
+    if (c->disc_mode != 0 && c->disc_mode != 1) return ROM_ERR_INVALID_ARG;
+    if ((int64_t)c->B * c->L >= (int64_t)1 << 30) return ROM_ERR_UNSUPPORTED;
+    if (c->B > 65535) return ROM_ERR_UNSUPPORTED;
+  }
+  if (which == 0) {
+    if (c->d_conv < 2 || c->d_conv > 4) return c->d_conv < 1 ? ROM_ERR_INVALID_ARG : ROM_ERR_UNSUPPORTED;
+    if (c->dt_rank < 1) return ROM_ERR_INVALID_ARG;
+    if (c->dtype == ROM_BF16 && c->dt_rank % 16 != 0) return ROM_ERR_UNSUPPORTED;
+    if (c->dtype == ROM_F32 && c->dt_rank % 4 != 0) return ROM_ERR_UNSUPPORTED;
+  }
+  return ROM_OK;
+}
+
+int check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ROM_ERR_CUDA;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ROM_ERR_CUDA;
+  return major == 10 ? ROM_OK : ROM_ERR_ARCH;
+}
+
+#define ROM_CUDA(expr)                            \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return ROM_ERR_CUDA;  \
+  } while (0)
+
+}  // namespace
+}  // namespace rom
+
+using namespace rom;
+
+extern "C" {
+
+int rom_workspace_size(const rom_config* cfg, size_t* bytes) {
+  if (!bytes) return ROM_ERR_INVALID_ARG;
+  // the layout is a function of the sizes only; fields a partial entry point ignores may be 0
+  if (!cfg || cfg->B < 1 || cfg->L < 1 || cfg->E < 1 || cfg->K < 1 || cfg->d_model < 0 || cfg->d_inner < 0 ||
+      cfg->dt_rank < 0 || cfg->d_state < 0 || (cfg->dtype != ROM_F32 && cfg->dtype != ROM_BF16))
+    return ROM_ERR_INVALID_ARG;
+  *bytes = make_layout(*cfg).total;
+  return ROM_OK;
+}
+
+int rom_workspace_find(const rom_config* cfg, const char* name, size_t* offset, size_t* bytes) {
+  if (!cfg || !name || !offset || !bytes) return ROM_ERR_INVALID_ARG;
+  const WsLayout l = make_layout(*cfg);
+  struct Item { const char* n; size_t off, sz; };
+  const Item items[] = {
+      {"U", l.U, l.esz * (size_t)l.T * cfg->d_inner},
+      {"delta_r", l.delta_r, l.esz * (size_t)l.T * cfg->dt_rank},
+      {"Bm", l.Bm, sizeof(float) * (size_t)l.T * cfg->d_state},
+      {"Cm", l.Cm, sizeof(float) * (size_t)l.T * cfg->d_state},
+      {"Delta", l.Delta, sizeof(float) * (size_t)l.T * cfg->d_inner},
+      {"row_of_assign", l.row_of_assign, sizeof(int32_t) * (size_t)l.A},
+      {"XZp", l.XZp, l.esz * (size_t)l.rows_max * 2 * cfg->d_inner},
+      {"Ygp", l.Ygp, l.esz * (size_t)l.rows_max * cfg->d_inner},
+      {"pad_offsets", l.pad_offsets, sizeof(int32_t) * (size_t)(cfg->E + 1)},
+  };
+  for (const Item& it : items)
+    if (std::strcmp(it.n, name) == 0) { *offset = it.off; *bytes = it.sz; return ROM_OK; }
+  return ROM_ERR_INVALID_ARG;
+}
+
+int rom_route(const rom_config* cfg, const void* x, const void* W_r, const float* b_r, int32_t* topk_idx, float* gates,
+              int32_t* counts, int32_t* offsets, int32_t* perm, int32_t* inv_perm, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg, 1);
+  if (rc != ROM_OK) return rc;
+  if (!x || !W_r || !ws) return ROM_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_r) || !aligned16(ws)) return ROM_ERR_INVALID_ARG;
+  const WsLayout lay = make_layout(*cfg);
+  if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
+  if ((rc = check_device()) != ROM_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LaunchCounter::count = 0;
+  ROM_CUDA(launch_route(*cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm, static_cast<char*>(ws), lay, st));
+  return ROM_OK;
+}
+
+int rom_scan(const rom_config* cfg, const void* u, const float* delta, const float* A, const float* Bm, const float* Cm,
+             const float* D, const void* z, const float* h0, void* y, float* h_last, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws; (void)ws_bytes;
+  int rc = check_config(cfg, 2);
+  if (rc != ROM_OK) return rc;
+  if (!u || !delta || !A || !Bm || !Cm || !y) return ROM_ERR_INVALID_ARG;
+  if (!aligned16(u) || !aligned16(delta) || !aligned16(A) || !aligned16(Bm) || !aligned16(Cm) || !aligned16(y) ||
+      (z && !aligned16(z)))
+    return ROM_ERR_INVALID_ARG;
+  if ((rc = check_device()) != ROM_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  LaunchCounter::count = 0;
+  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, h0, y, h_last, nullptr, 1, st));
+  return ROM_OK;
+}
+
+int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
+                      float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg, 0);
+  if (rc != ROM_OK) return rc;
+  if (!w || !x || !out || !ws) return ROM_ERR_INVALID_ARG;
+  if (!w->W_r || !w->W_inz || !w->w_conv || !w->W_x || !w->W_dt || !w->A || !w->W_out) return ROM_ERR_INVALID_ARG;
+  const void* ptrs[] = {x, out, ws, w->W_r, w->W_inz, w->w_conv, w->W_x, w->W_dt, w->A, w->W_out};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return ROM_ERR_INVALID_ARG;
+  const rom_config& c = *cfg;
+  const WsLayout lay = make_layout(c);
+  if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
+  if ((rc = check_device()) != ROM_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* W = static_cast<char*>(ws);
+  LaunchCounter::count = 0;
+
+  const int T = (int)lay.T, De = c.d_inner, Dm = c.d_model, R = c.dt_rank, N = c.d_state;
+  const bool tc = c.dtype == ROM_BF16 && !(c.flags & ROM_FLAG_SIMT_GEMM);
+  int32_t* status = reinterpret_cast<int32_t*>(W + lay.status);
+  int32_t* tile_expert = reinterpret_cast<int32_t*>(W + lay.tile_expert);
+  int32_t* num_m_tiles = reinterpret_cast<int32_t*>(W + lay.num_m_tiles);
+  int32_t* row_of_assign = reinterpret_cast<int32_t*>(W + lay.row_of_assign);
+  float* gates = gates_out ? gates_out : reinterpret_cast<float*>(W + lay.gates);
+
+  ROM_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t) * kStatusInts, st));
+  // S1 + S2: router, top-K, permutation tables
+  ROM_CUDA(launch_route(c, x, w->W_r, w->b_r, topk_idx_out, gates, counts_out, nullptr, nullptr, nullptr, W, lay, st));
+  ROM_CUDA(launch_gather_rows(c, x, W, lay, st));
+
+  auto gemm = [&](const void* A_, int lda, const void* B_, int ldb, int n_experts, int64_t bstride, int M_max, int Nn, int Kd,
+                  const int32_t* te, const int32_t* nmt, const Epilogue& ep) -> cudaError_t {
+    if (tc) return launch_gemm_tc(A_, lda, B_, ldb, n_experts, M_max, Nn, Kd, te, nmt, ep, status, st);
+    return launch_gemm_simt(c.dtype, A_, lda, B_, ldb, bstride, M_max, Nn, Kd, te, nmt, ep, st);
+  };
+
+  // S3: grouped [Conv Proj | Gate Proj]
+  Epilogue e_in{EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, 0, 0};
+  ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
+  // S4: un-permute + sum over selected experts + conv + SiLU
+  ROM_CUDA(launch_conv(c, W + lay.XZp, row_of_assign, w->w_conv, w->b_conv, W + lay.U, st));
+  // S5: x Proj -> delta_r | B | C
+  Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N};
+  ROM_CUDA(gemm(W + lay.U, De, w->W_x, De, 1, 0, T, R + 2 * N, De, nullptr, nullptr, e_x));
+  // S6: dt Proj + softplus
+  Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0};
+  ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
+  // S7 + S8 + S9: scan, gate, re-permute
+  const char* zbase = W + lay.XZp + (size_t)De * lay.esz;
+  ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
+                       reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, 2 * De, nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, st));
+  // S10: grouped Out Proj
+  Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0};
+  ROM_CUDA(gemm(W + lay.Ygp, De, w->W_out, De, c.E, (int64_t)Dm * De, (int)lay.rows_max, Dm, De, tile_expert, num_m_tiles, e_out));
+  // S11: gate-weighted combine
+  ROM_CUDA(launch_combine(c, W + lay.Op, row_of_assign, gates, out, st));
+  return ROM_OK;
+}
+
+int rom_get_status(void* ws, void* stream, int32_t* host_code) {
+  if (!ws || !host_code) return ROM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t v[2] = {0, 0};
+  ROM_CUDA(cudaMemcpyAsync(v, ws, sizeof(v), cudaMemcpyDeviceToHost, st));
+  ROM_CUDA(cudaStreamSynchronize(st));
+  ROM_CUDA(cudaMemsetAsync(ws, 0, sizeof(int32_t) * kStatusInts, st));
+  *host_code = v[kStatCode] == 0 ? ROM_OK : ROM_ERR_DEVICE_TIMEOUT;
+  return ROM_OK;
+}
+
+const char* rom_status_string(int code) {
+  switch (code) {
+    case ROM_OK: return "ok";
+    case ROM_ERR_INVALID_ARG: return "invalid argument";
+    case ROM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case ROM_ERR_WORKSPACE: return "workspace too small";
+    case ROM_ERR_CUDA: return "CUDA call failed";
+    case ROM_ERR_ARCH: return "device is not sm_100";
+    case ROM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+int rom_last_launch_count(void) { return LaunchCounter::count; }
+
+}  // extern "C"

@@ -1,0 +1,353 @@
+// bf16 grouped GEMM on the 5th-generation tensor cores (tcgen05 + TMEM), operands staged by TMA.
+//
+//   C[M, N] = A[M, Kd] * B[e(m)][N, Kd]^T,  fp32 accumulation in tensor memory.
+//
+// A holds token rows grouped by expert, every expert segment padded to a multiple of the 128-row
+// tile, so a row tile never straddles two experts and a device-built table gives the expert of each
+// row tile; the number of row tiles is read from device memory (no host synchronisation).  This is
+// the per-expert Conv/Gate projection and Out projection of Section 4.2 (dropless, Section 5.1); with
+// one "expert" it also serves the shared x Proj / dt Proj.
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0      TMA producer: A tile 128x64 and B tile block_n x 64 per stage, 128-byte swizzle
+//   warp 1      allocates TMEM, issues tcgen05.mma (one thread), commits to mbarriers
+//   warps 2..5  epilogue: tcgen05.ld of the 128 x block_n fp32 accumulator, fused output op, stores
+// The accumulator is double-buffered in TMEM (2 x 256 columns) so the epilogue of tile i overlaps
+// the MMAs of tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches an error code in
+// the status word, drains its own copies with a bounded wait, frees its TMEM and returns.
+//
+// No cluster multicast is used anywhere in this file.
+#include <cuda.h>
+
+#include "rom_internal.cuh"
+
+namespace rom {
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;            // 64 bf16 = 128 bytes = one swizzle row
+constexpr int MAX_BLOCK_N = 256;
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;          // 16 KB
+constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;      // 32 KB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int ACC_STAGES = 2;
+constexpr int TMEM_COLS = 512;
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait polls before a wait gives up (a few seconds)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit is reached or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements),
+// written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset),
+// the leading byte offset is unused for swizzled K-major layouts, descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);          // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                            // leading byte offset (ignored)
+  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+  d |= (uint64_t)1 << 46;                            // version
+  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+  return d;
+}
+
+// Fused output op on one row segment of 8 consecutive columns (n0 % 8 == 0).
+__device__ __forceinline__ void epi_store8(const Epilogue& ep, size_t m, int n0, const float (&v)[8]) {
+  if (ep.mode == EPI_STORE || (ep.mode == EPI_XPROJ && n0 < ep.R)) {
+    const int ld = ep.mode == EPI_STORE ? ep.ldc : ep.R;
+    uint4 q;
+    uint32_t* w = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + m * ld + n0) = q;
+  } else if (ep.mode == EPI_XPROJ) {
+    float* dst = (n0 < ep.R + ep.N) ? ep.Bm + m * ep.N + (n0 - ep.R) : ep.Cm + m * ep.N + (n0 - ep.R - ep.N);
+    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+  } else {
+    float o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = softplus_f(v[i] + (ep.bias ? __ldg(ep.bias + n0 + i) : 0.0f));
+    float* dst = reinterpret_cast<float*>(ep.C) + m * ep.ldc + n0;
+    *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+    *reinterpret_cast<float4*>(dst + 4) = make_float4(o[4], o[5], o[6], o[7]);
+  }
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               int M_max, int N, int Kd, int block_n, uint32_t idesc,
+               const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ num_m_tiles_dev,
+               Epilogue ep, int32_t* __restrict__ status) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;               // 128B-swizzled tiles need 1024-byte alignment
+  unsigned char* smem = smem_raw + (base - raw);
+  const uint32_t bars = base + STAGES * STAGE_BYTES;          // barrier block (8-byte aligned)
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + ACC_STAGES + a); };
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2 * ACC_STAGES));
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  int num_m_tiles = (M_max + BLOCK_M - 1) / BLOCK_M;
+  if (num_m_tiles_dev) num_m_tiles = min(num_m_tiles, *num_m_tiles_dev);
+  const int M_valid = min(M_max, num_m_tiles * BLOCK_M);
+  const int n_tiles = (N + block_n - 1) / block_n;
+  const int total_tiles = num_m_tiles * n_tiles;
+  const int num_kb = (Kd + BLOCK_K - 1) / BLOCK_K;
+  const uint32_t stage_tx = A_STAGE_BYTES + (uint32_t)block_n * BLOCK_K * 2;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int issued = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m_tile = tile / n_tiles, n_tile = tile % n_tiles;
+        const int e = tile_expert ? tile_expert[m_tile] : 0;
+        const int b_row = e * N + n_tile * block_n;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(full_bar(stage), stage_tx);
+          const uint32_t sa = base + stage * STAGE_BYTES;
+          tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BLOCK_K, m_tile * BLOCK_M);
+          tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row);
+          ++issued;
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        if (!*abort_flag) { atomicExch(status + kStatCode, ROM_ERR_DEVICE_TIMEOUT); atomicExch(status + kStatWhere, 1); }
+        *abort_flag = 1;
+      }
+      if (*abort_flag) {
+        // drain: give this CTA's copies still in flight a bounded time to land before the CTA exits
+        int s = stage; uint32_t ph = phase;
+        for (int i = 0; i < min(issued, STAGES); ++i) {
+          if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
+          for (uint32_t it = 0; it < (1u << 20); ++it)
+            if (mbar_try_wait(full_bar(s), ph)) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + (uint32_t)acc * MAX_BLOCK_N;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + stage * STAGE_BYTES;
+          const uint64_t adesc = make_smem_desc(sa);
+          const uint64_t bdesc = make_smem_desc(sa + A_STAGE_BYTES);
+#pragma unroll
+          for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+            // advance 16 elements = 32 bytes along K inside the swizzled row: +2 in the address field
+            umma_bf16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));
+        if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) {
+        if (!*abort_flag) { atomicExch(status + kStatCode, ROM_ERR_DEVICE_TIMEOUT); atomicExch(status + kStatWhere, 2); }
+        *abort_flag = 1;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const int m_tile = tile / n_tiles, n_tile = tile % n_tiles;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int row = m_tile * BLOCK_M + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * MAX_BLOCK_N;
+      for (int c0 = 0; c0 < block_n; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c0, r);
+        if (row < M_valid) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 8) {
+            const int n0 = n_tile * block_n + c0 + j;
+            if (n0 < N) {
+              float v[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j + i]);
+              epi_store8(ep, (size_t)row, n0, v);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (!ok && lane == 0) {
+      if (!*abort_flag) { atomicExch(status + kStatCode, ROM_ERR_DEVICE_TIMEOUT); atomicExch(status + kStatWhere, 3); }
+      *abort_flag = 1;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;      // resolving the driver symbol is idempotent; a benign race
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(p);
+  return fn;
+}
+
+// 2-D bf16 row-major [rows, cols] (cols contiguous, row stride ld elements); box = 64 cols x box_rows.
+bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {BLOCK_K, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int n_experts, int M_max, int N, int Kd,
+                           const int32_t* tile_expert, const int32_t* num_m_tiles_dev, const Epilogue& epi,
+                           int32_t* status, cudaStream_t st) {
+  // N tile: a multiple of 32 (epilogue column groups) and of 16 (UMMA N for M = 128), at most 256
+  int block_n = N >= MAX_BLOCK_N ? MAX_BLOCK_N : (N + 31) / 32 * 32;
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, A, (uint64_t)M_max, (uint64_t)Kd, (uint64_t)lda, BLOCK_M)) return cudaErrorInvalidValue;
+  if (!make_tmap(&tb, Bw, (uint64_t)n_experts * N, (uint64_t)Kd, (uint64_t)ldb, (uint32_t)block_n)) return cudaErrorInvalidValue;
+  // instruction descriptor: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
+  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+  }
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int n_tiles = (N + block_n - 1) / block_n;
+  const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
+  const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
+  gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace rom

@@ -1,0 +1,97 @@
+// Internal declarations shared by the CUDA translation units of the RoM forward library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rom.h"
+
+namespace rom {
+
+constexpr int kTileM = 128;        // expert segments are padded to this many rows (GEMM M tile)
+constexpr int kChunkTokens = 32;   // tokens per routing chunk (one warp)
+constexpr int kMaxE = 64;
+constexpr int kMaxK = 8;
+constexpr int kStatusInts = 64;    // status block at the head of the workspace
+
+// status word slots
+constexpr int kStatCode = 0;       // 0 or ROM_ERR_DEVICE_TIMEOUT
+constexpr int kStatWhere = 1;      // which wait gave up (debug aid)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Workspace carving, identical for every entry point (host arithmetic only).
+struct WsLayout {
+  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts;
+  size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
+  size_t x_perm, XZp, U, delta_r, Bm, Cm, Delta, Ygp, Op;
+  size_t total;
+  int64_t T, A, rows_max, max_m_tiles, n_chunks;
+  size_t esz;
+};
+WsLayout make_layout(const rom_config& c);
+
+struct LaunchCounter { static thread_local int count; };
+inline void count_launch() { LaunchCounter::count++; }
+
+// ---------------------------------------------------------------- epilogues shared by both GEMM paths
+enum EpiMode : int {
+  EPI_STORE = 0,      // C[m, n] = acc                          (dtype)
+  EPI_XPROJ = 1,      // n < R: delta_r[m, n] (dtype); then Bm[m, n-R], Cm[m, n-R-N] (fp32)
+  EPI_SOFTPLUS = 2    // Delta[m, n] = softplus(acc + bias[n])  (fp32)
+};
+struct Epilogue {
+  int mode;
+  void* C;            // EPI_STORE: [M, ldc] dtype;  EPI_XPROJ: delta_r [M, R] dtype;  EPI_SOFTPLUS: float [M, ldc]
+  int ldc;
+  float* Bm;          // EPI_XPROJ
+  float* Cm;
+  const float* bias;  // EPI_SOFTPLUS (may be null)
+  int R, N;
+};
+
+// ---------------------------------------------------------------- launchers (each returns a cudaError_t)
+cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, const float* b_r,
+                         int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
+                         int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st);
+
+cudaError_t launch_gather_rows(const rom_config& c, const void* x, char* ws, const WsLayout& lay, cudaStream_t st);
+
+// C[M,N] = A[M,Kd] * B[e][N,Kd]^T, A and B K-contiguous.  Grouped when tile_expert != nullptr: row tile
+// i (kTileM rows) uses expert tile_expert[i]; the number of valid row tiles is *num_m_tiles_dev.
+cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* Bw, int ldb, int64_t b_expert_stride,
+                             int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
+                             const Epilogue& epi, cudaStream_t st);
+
+cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int n_experts,
+                           int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
+                           const Epilogue& epi, int32_t* status, cudaStream_t st);
+
+cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
+                        const float* b_conv, void* U, cudaStream_t st);
+
+// Scan.  row_map == nullptr: y is [T, d_inner] and z is [T, ldz]; otherwise y row of (t, k) is
+// row_map[t*K + k] (K rows written per token) and z is read from row row_map[t*K + k] of a
+// [rows, ldz] matrix and summed over k.
+cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
+                        const float* Cm, const float* D, const void* z, int ldz, const float* h0, void* y,
+                        float* h_last, const int32_t* row_map, int K, cudaStream_t st);
+
+cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,
+                           void* out, cudaStream_t st);
+
+// ---------------------------------------------------------------- device helpers
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
+__device__ __forceinline__ float softplus_f(float v) {
+  // max(v,0) + log1p(exp(-|v|)); log1pf keeps relative accuracy when exp(-|v|) is tiny
+  return fmaxf(v, 0.0f) + log1pf(__expf(-fabsf(v)));
+}
+
+}  // namespace rom

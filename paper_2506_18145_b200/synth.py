@@ -53,7 +53,7 @@ CONFIGS: Dict[str, RomShape] = {
     "small_bf16": RomShape("small_bf16", 4, 2048, 1024, 2048, 16, 4, 64, 8, 1, "bf16", 2000),
     "long_ctx": RomShape("long_ctx", 1, 16384, 2048, 4096, 16, 4, 128, 8, 1, "bf16", 3000),
     "zipf": RomShape("zipf", 8, 4096, 2048, 4096, 16, 4, 128, 16, 2, "bf16", 4000,
-                     router_bias_scale=1.0),
+                     router_bias_scale=0.657),
     "short_seqs": RomShape("short_seqs", 64, 1024, 1536, 3072, 16, 4, 96, 8, 2, "bf16", 5000),
 }
 

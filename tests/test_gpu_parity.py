@@ -1,0 +1,186 @@
+"""Parity of the CUDA path (called through the C ABI) against the CPU fp64 oracle on the same
+seeded inputs.  Integer results (top-K indices, counts, offsets, permutation) must be bit-exact;
+floating-point results within 1e-4 (fp32 path) / 2e-2 (bf16 path) relative, in max-norm and 2-norm."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rom_oracle as O
+from paper_2506_18145_b200 import binding as rb
+from paper_2506_18145_b200 import synth
+
+from rom_testlib import TOL, GpuLayer, assert_close, check_route_exact, gpu_route, np64, oracle_layer
+
+pytestmark = pytest.mark.gpu
+
+
+def small_shape(**kw):
+    base = dict(name="t", B=2, L=300, d_model=128, d_inner=256, d_state=16, d_conv=4, dt_rank=16, E=4, K=2,
+                dtype="bf16", seed_base=77000)
+    base.update(kw)
+    return synth.RomShape(**base)
+
+
+# ---------------------------------------------------------------------------------------------- routing
+@pytest.mark.parametrize("kw", [
+    dict(B=1, L=50, E=5, K=2),                       # one ragged chunk
+    dict(B=3, L=333, E=8, K=1),                      # ragged tail, several blocks
+    dict(B=2, L=1000, E=16, K=2),
+    dict(B=1, L=257, E=64, K=8, d_model=64),         # maximum E and K
+    dict(B=1, L=1, E=3, K=3),                        # a single token, K = E
+    dict(B=4, L=512, E=8, K=2, dtype="f32"),
+    dict(B=1, L=4096, E=1, K=1),                     # one expert
+])
+@pytest.mark.parametrize("gate_mode", [0, 1])
+def test_route_bit_exact(kw, gate_mode):
+    s = small_shape(**kw)
+    p = synth.make_inputs(s, recipe="unit")
+    got = gpu_route(s, p, gate_mode)
+    check_route_exact(got, s, p, gate_mode)
+
+
+def test_route_ties_bias_and_empty_experts():
+    s = small_shape(B=2, L=200, E=8, K=2, router_bias_scale=3.0)
+    p = synth.make_inputs(s, recipe="unit")
+    W = p["W_r"].clone(); W[5] = W[2]; W[7] = 0; p["W_r"] = W          # duplicate rows: ties -> lowest id
+    b = p["b_r"].clone(); b[5] = b[2]; b[6] = -1e9; p["b_r"] = b        # expert 6 never chosen
+    got = gpu_route(s, p)
+    idx, _ = check_route_exact(got, s, p)
+    assert got["counts"][6] == 0
+    assert not np.any(idx[:, 0] == 5)          # the duplicate of expert 2 never comes first
+    # all-zero tokens: every logit equals the bias; without bias -> experts 0..K-1
+    p2 = synth.make_inputs(small_shape(B=1, L=70, E=6, K=3), recipe="unit")
+    p2["x"] = torch.zeros_like(p2["x"])
+    s2 = small_shape(B=1, L=70, E=6, K=3)
+    got2 = gpu_route(s2, p2)
+    check_route_exact(got2, s2, p2)
+    assert np.array_equal(got2["idx"], np.tile(np.arange(3, dtype=np.int32), (70, 1)))
+
+
+@pytest.mark.parametrize("name", ["tiny_fp32", "small_bf16", "long_ctx", "zipf", "short_seqs"])
+def test_route_bit_exact_full_size_configs(name):
+    s = synth.CONFIGS[name]
+    small = s.replace(d_inner=64, dt_rank=16)       # x, W_r, b_r depend only on the seeds and d_model
+    p = synth.make_inputs(small)
+    got = gpu_route(s, p)
+    check_route_exact(got, s, p)
+    if name == "zipf":
+        ratio = got["counts"].max() / got["counts"].mean()
+        assert 4.5 < ratio < 5.5, ratio
+
+
+# ---------------------------------------------------------------------------------------------- scan
+def run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed):
+    q = synth.make_scan_inputs(B, L, De, 16, dtype, seed, with_z=with_z, with_h0=with_h0)
+    if not with_D:
+        q["D"] = None
+    cfg = rb.make_config(B, L, 64, De, 16, 4, 16, 1, 1, dtype, 0, disc_mode)
+    d = {k: (None if v is None else v.cuda()) for k, v in q.items()}
+    y = torch.empty_like(d["u"])
+    h_last = torch.empty((B, De, 16), dtype=torch.float32, device="cuda")
+    rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], d["h0"], y, h_last)
+    torch.cuda.synchronize()
+    Y, hl = O.selective_scan(np64(q["u"]), np64(q["delta"]), np64(q["A"]), np64(q["Bm"]), np64(q["Cm"]), np64(q["D"]),
+                             np64(q["h0"]), disc_mode)
+    if with_z:
+        Y = O.gated(Y, np64(q["z"]))
+    return np64(y), Y, np64(h_last), hl
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("disc_mode", [0, 1])
+@pytest.mark.parametrize("B,L,De,with_z,with_h0,with_D", [
+    (2, 100, 192, True, False, True),      # ragged L, channel count not a multiple of the block
+    (1, 777, 64, False, True, False),      # no gate, initial state, no skip
+    (3, 1, 128, True, True, True),         # single step
+    (1, 2048, 256, True, False, True),     # several time tiles
+])
+def test_scan_parity(dtype, disc_mode, B, L, De, with_z, with_h0, with_D):
+    y, Y, hl, HL = run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed=9100 + L)
+    assert_close(y, Y, TOL[dtype], "scan y")
+    assert_close(hl, HL, 1e-4 if dtype == "f32" else 2e-3, "scan h_last")
+
+
+def test_scan_long_memory_small_delta():
+    # Delta*A down to -1e-3: the regime where exp(x) - 1 cancels; the fp32 path must still hold 1e-4
+    B, L, De = 1, 4096, 64
+    q = synth.make_scan_inputs(B, L, De, 16, "f32", 9300, with_z=False)
+    q["delta"] = q["delta"] * 0.05
+    q["A"] = -torch.ones_like(q["A"]) * torch.linspace(0.2, 1.0, 16)[None, :]
+    cfg = rb.make_config(B, L, 64, De, 16, 4, 16, 1, 1, "f32")
+    d = {k: (None if v is None else v.cuda()) for k, v in q.items()}
+    y = torch.empty_like(d["u"])
+    rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], None, None, y, None)
+    torch.cuda.synchronize()
+    Y, _ = O.selective_scan(np64(q["u"]), np64(q["delta"]), np64(q["A"]), np64(q["Bm"]), np64(q["Cm"]), np64(q["D"]))
+    assert_close(np64(y), Y, 1e-4, "long-memory scan")
+
+
+# ---------------------------------------------------------------------------------------------- layer
+def check_layer(s, recipe, with_D=True, gate_mode=0, disc_mode=0, flags=0, check_taps=True):
+    p = synth.make_inputs(s, recipe=recipe, with_D=with_D)
+    ref, im = oracle_layer(s, p, gate_mode, disc_mode)
+    g = GpuLayer(s, p, gate_mode, disc_mode, flags)
+    out = g.forward()
+    tol = TOL[s.dtype]
+    np.testing.assert_array_equal(g.idx.cpu().numpy(), im["idx"])
+    np.testing.assert_array_equal(g.counts.cpu().numpy(), im["counts"])
+    np.testing.assert_allclose(g.gates.cpu().numpy(), im["gate"], rtol=2e-6)
+    if check_taps:
+        tdt = synth.torch_dtype(s)
+        assert_close(np64(g.tap("U", tdt, s.d_inner)), im["U"], tol, "U")
+        assert_close(np64(g.tap("Bm", torch.float32, s.d_state)), im["Bm"], tol, "Bm")
+        assert_close(np64(g.tap("Cm", torch.float32, s.d_state)), im["Cm"], tol, "Cm")
+        assert_close(np64(g.tap("Delta", torch.float32, s.d_inner)), im["Delta"], tol, "Delta")
+        rows = g.tap("row_of_assign", torch.int32, 1).view(-1)[::s.K].long()      # slot 0 row of each token
+        assert_close(np64(g.tap("Ygp", tdt, s.d_inner)[rows]), im["Yg"], tol, "Yg")
+    e = assert_close(np64(out), ref, tol, "out")
+    assert rb.last_launch_count() >= 9
+    return e
+
+
+@pytest.mark.parametrize("recipe,with_D", [("paper", True), ("unit", True), ("unit", False)])
+def test_layer_tiny_fp32_config(recipe, with_D):
+    check_layer(synth.CONFIGS["tiny_fp32"], recipe, with_D)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),                                                       # K = 2, ragged L
+    dict(E=8, K=1, B=3, L=130),
+    dict(E=3, K=3, L=64, d_conv=3),
+    dict(E=4, K=1, d_conv=2, dt_rank=32, B=1, L=1),               # one token
+    dict(E=6, K=2, router_bias_scale=4.0, L=513),                 # skewed loads, some experts nearly empty
+])
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
+def test_layer_small_shapes(kw, dtype, flags):
+    s = small_shape(dtype=dtype, **kw)
+    check_layer(s, "unit", flags=flags)
+
+
+@pytest.mark.parametrize("gate_mode,disc_mode", [(1, 0), (0, 1), (1, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_layer_modes(gate_mode, disc_mode, dtype):
+    s = small_shape(dtype=dtype, L=200)
+    check_layer(s, "unit", gate_mode=gate_mode, disc_mode=disc_mode)
+
+
+def test_layer_single_expert_is_dense_mamba_on_gpu():
+    s = small_shape(E=1, K=1, L=256, dtype="bf16")
+    check_layer(s, "unit")
+
+
+@pytest.mark.parametrize("recipe,with_D", [("paper", True), ("unit", False)])
+def test_layer_small_bf16_config(recipe, with_D):
+    check_layer(synth.CONFIGS["small_bf16"], recipe, with_D)
+
+
+def test_layer_batch_permutation_invariance_on_gpu():
+    s = small_shape(B=4, L=128, E=4, K=2)
+    p = synth.make_inputs(s, recipe="unit")
+    g = GpuLayer(s, p)
+    out = g.forward().clone()
+    counts = g.counts.clone()
+    pi = torch.tensor([2, 0, 3, 1], device="cuda")
+    out2 = g.forward(g.dev["x"][pi].contiguous())
+    assert torch.equal(out2, out[pi])
+    assert torch.equal(g.counts, counts)
