@@ -1,0 +1,320 @@
+#!/usr/bin/env python
+"""Benchmark of the RoM layer forward on B200: tokens/s of one full pass of the hot path
+(route -> permute -> grouped Conv/Gate Proj -> conv1d+SiLU -> x/dt Proj -> scan -> gate ->
+grouped Out Proj -> combine) on a seeded synthetic workload, with a per-kernel roofline and the
+CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl reference]
+
+Prints ONE JSON line on rank 0.  With --gpus N > 1 (launched under torchrun, one rank per GPU) every
+rank runs an independent replica of the same workload (the forward has no exchange step: routing is
+per token, conv and scan per sequence), timing is the max over ranks, value is the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2506_18145_b200 import synth  # noqa: E402
+
+METRIC = "RoM layer fwd tokens/sec"
+UNIT = "tokens/s"
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from one
+# ncu capture, keyed by (stage, workload); None = not captured.  The summaries the figures come from
+# are the text files under profiles/.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def algorithmic_work(s: synth.RomShape):
+    """Per launch: flops of the tensor-bound stages, bytes of the HBM-bound ones (bf16 storage = 2 B).
+    Padding rows, workspace re-reads and fp32 storage of Delta are NOT counted (algorithmic, not moved)."""
+    T, A = s.T, s.T * s.K
+    esz = 2 if s.dtype == "bf16" else 4
+    Dm, De, N, R = s.d_model, s.d_inner, s.d_state, s.dt_rank
+    return {
+        "route": ("hbm", T * Dm * esz + 16 * A),
+        "gather": ("hbm", 2 * A * Dm * esz),
+        "in_proj": ("tensor", 2.0 * A * Dm * 2 * De),
+        "conv": ("hbm", (s.K + 1) * T * De * esz),
+        "x_proj": ("hbm", T * De * esz + T * (R * esz + 2 * N * 4)),
+        "dt_proj": ("hbm", T * R * esz + T * De * esz),
+        "scan": ("hbm", T * (4 * De * esz + 8 * N)),
+        "out_proj": ("tensor", 2.0 * A * De * Dm),
+        "combine": ("hbm", (s.K + 1) * T * Dm * esz),
+    }
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clock and throttle reasons during the timed region."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.tmp.close()
+        try:
+            os.unlink(self.tmp.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample(s: synth.RomShape, p, n_tokens: int):
+    """Run the CPU oracle, as it stands, on the first n_tokens of sequence 0 (the layer is causal, so
+    this is the same workload's prefix).  Returns (seconds, tokens, threads)."""
+    import numpy as np
+    from oracle import rom_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    f = lambda v: None if v is None else v.double().numpy()
+    Ls = min(n_tokens, s.L)
+    x = f(p["x"][:1, :Ls])
+    args = [f(p[k]) for k in ("W_r", "b_r", "W_inz", "w_conv", "b_conv", "W_x", "W_dt", "b_dt", "A", "D", "W_out")]
+    t0 = time.perf_counter()
+    O.rom_layer_forward(x, *args, K=s.K, dt_rank=s.dt_rank)
+    return time.perf_counter() - t0, Ls, threads
+
+
+def run_reference(args, s):
+    """--impl reference: the CPU oracle timed on the host cores, each step a bounded prefix sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    p = synth.make_inputs(s)
+    n_tok = min(s.L, 1024)
+    for _ in range(args.warmup):
+        oracle_sample(s, p, min(n_tok, 256))
+    times = []
+    threads = 1
+    for _ in range(args.steps):
+        dt, ntok, threads = oracle_sample(s, p, n_tok)
+        times.append(dt)
+    total = sum(times)
+    value = n_tok * args.steps / total
+    sample = f"first {n_tok} tokens of sequence 0 of {s.name} per step (causal prefix of the same workload)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(s),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(s):
+    return {"workload": s.name, "B": s.B, "L": s.L, "d_model": s.d_model, "d_inner": s.d_inner, "d_state": s.d_state,
+            "d_conv": s.d_conv, "dt_rank": s.dt_rank, "E": s.E, "K": s.K, "storage": s.dtype,
+            "l2": "inputs+weights larger than L2 (no flush between iterations)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="long_ctx", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--simt", action="store_true", help="run the projections on the fp32-FMA bisecting path")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    s = synth.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        run_reference(args, s)
+        return
+
+    from paper_2506_18145_b200 import binding as rb
+    rb.lib()                                  # fail loudly if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+
+    p = synth.make_inputs(s)
+    d = {k: (None if v is None else v.to(dev)) for k, v in p.items()}
+    cfg = rb.config_from_shape(s, flags=rb.ROM_FLAG_SIMT_GEMM if args.simt else 0)
+    weights = rb.make_weights(d)
+    ws = rb.alloc_workspace(cfg, dev)
+    x_dev = d["x"]
+    out = torch.empty_like(x_dev)
+    x_host = p["x"].pin_memory()
+    out_host = torch.empty_like(p["x"]).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        rb.rom_layer_forward(cfg, weights, x_dev, out, None, None, None, ws, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    code = rb.rom_get_status(ws)
+    if code != 0:
+        raise SystemExit("device status: " + rb.status_string(code))
+    launches_per_step = rb.last_launch_count()
+
+    # ---- timed region: K steps, inputs resident in HBM
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+
+    # ---- end to end: host buffers, H2D of x and D2H of out inside the timed region
+    for _ in range(2):
+        x_dev.copy_(x_host, non_blocking=True); step(); out_host.copy_(out, non_blocking=True)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(args.steps):
+        x_dev.copy_(x_host, non_blocking=True)
+        step()
+        out_host.copy_(out, non_blocking=True)
+    f1.record(stream)
+    barrier()
+    ms_e2e = f0.elapsed_time(f1)
+
+    if dist is not None:
+        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+
+    # ---- per-stage device times (CUDA events between the kernels, same stream, same inputs)
+    stage_ms = {}
+    if rank == 0:
+        acc = {}
+        n_prof = max(3, min(args.steps, 10))
+        for _ in range(n_prof):
+            for k, v in rb.rom_layer_forward_profile(cfg, weights, x_dev, out, ws, stream).items():
+                acc.setdefault(k, []).append(v)
+        stage_ms = {k: sum(v) / len(v) for k, v in acc.items()}
+    code = rb.rom_get_status(ws)
+    if code != 0:
+        raise SystemExit("device status: " + rb.status_string(code))
+
+    if rank == 0:
+        peaks = load_peaks()
+        work = algorithmic_work(s)
+        kernels = {}
+        for name, t_ms in stage_ms.items():
+            bound, amount = work[name]
+            if bound == "tensor":
+                ach = amount / (t_ms * 1e-3) / 1e12
+                peak, unit = peaks["bf16_tflops"], "TFLOP/s"
+            else:
+                ach = amount / (t_ms * 1e-3) / 1e9
+                peak, unit = peaks["hbm_gbs"], "GB/s"
+            kernels[name] = {"ms": round(t_ms, 4), "bound": bound, "achieved": round(ach, 2), "peak": peak, "unit": unit,
+                             "frac": round(ach / peak, 4)}
+        dom = max(stage_ms, key=stage_ms.get)
+        k = kernels[dom]
+        roofline = {"kernel": dom, "bound": k["bound"], "achieved": k["achieved"], "peak": k["peak"], "unit": k["unit"],
+                    "frac": k["frac"], "traffic": NCU_TRAFFIC_BYTES.get((dom, s.name)),
+                    "peak_source": f"of {peaks['source']} (burst bf16 / copy bandwidth)",
+                    "how": "CUDA events between stages on the launch stream, mean over profiled steps"}
+        # MUFU view of the scan: one ex2 per (token, channel, state) against 16 lanes/clk/SM * 148 SMs
+        if "scan" in stage_ms and clocks and clocks.get("sm_max_mhz"):
+            exps = s.T * s.d_inner * s.d_state
+            peak_exps = 148 * 16 * clocks["sm_max_mhz"] * 1e6
+            kernels["scan"]["alu_mufu_frac"] = round(exps / (stage_ms["scan"] * 1e-3) / peak_exps, 4)
+
+        tokens = s.T * world
+        cpu = None
+        if not args.no_cpu_baseline:
+            n_tok = min(s.L, 4096)
+            dt, ntok, threads = oracle_sample(s, p, n_tok)
+            cpu = {"value": ntok / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                   "sample": f"first {ntok} tokens of sequence 0 of {s.name}, one run ({dt:.1f} s)"}
+        line = {"metric": METRIC, "value": tokens * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic",
+                "config": workload_config(s), "clocks": clocks,
+                "e2e": {"value": tokens * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+                        "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
+                        "d2h_bytes_per_step": out_host.numel() * out_host.element_size()},
+                "gpu_launches": launches_per_step * args.steps,
+                "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

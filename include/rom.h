@@ -118,6 +118,15 @@ ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const
                       int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
                       void *ws, size_t ws_bytes, void *stream);
 
+/* Profiling aid: the same launch sequence as rom_layer_forward with a CUDA event recorded on
+ * `stream` between stages; synchronises the stream and writes the device time of each stage in
+ * milliseconds to stage_ms (host out, at least rom_num_stages() floats).  Stage i is named
+ * rom_stage_name(i): route, gather, in_proj, conv, x_proj, dt_proj, scan, out_proj, combine.      */
+ROM_API int rom_layer_forward_profile(const rom_config *cfg, const rom_weights *w, const void *x, void *out,
+                              void *ws, size_t ws_bytes, void *stream, float *stage_ms, int n_stage_ms);
+ROM_API int rom_num_stages(void);
+ROM_API const char *rom_stage_name(int i);
+
 /* Locate a named intermediate of the last rom_layer_forward inside the workspace (host-only
  * arithmetic; for tests and debugging).  Names: "U" [T,D_e] dtype, "delta_r" [T,d_r] dtype,
  * "Bm","Cm" [T,D_s] f32, "Delta" [T,D_e] f32, "row_of_assign" [T*K] i32 (padded row of each

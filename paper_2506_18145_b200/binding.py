@@ -20,7 +20,8 @@ ROM_FLAG_SIMT_GEMM = 1
 ROM_OK = 0
 
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
-           "rom_get_status", "rom_status_string", "rom_last_launch_count")
+           "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
+           "rom_num_stages", "rom_stage_name")
 
 
 class RomConfig(ctypes.Structure):
@@ -62,8 +63,13 @@ def lib() -> ctypes.CDLL:
         L.rom_status_string.argtypes = [ctypes.c_int]
         L.rom_status_string.restype = ctypes.c_char_p
         L.rom_last_launch_count.argtypes = []
+        L.rom_layer_forward_profile.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, vp, ctypes.c_size_t, vp,
+                                                ctypes.POINTER(ctypes.c_float), ctypes.c_int]
+        L.rom_num_stages.argtypes = []
+        L.rom_stage_name.argtypes = [ctypes.c_int]
+        L.rom_stage_name.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name != "rom_status_string":
+            if name not in ("rom_status_string", "rom_stage_name"):
                 getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -156,3 +162,20 @@ def rom_get_status(ws, stream=None) -> int:
 
 def last_launch_count() -> int:
     return int(lib().rom_last_launch_count())
+
+
+def stage_names():
+    L = lib()
+    return [L.rom_stage_name(i).decode() for i in range(L.rom_num_stages())]
+
+
+def rom_layer_forward_profile(cfg, weights: RomWeights, x, out, ws, stream=None):
+    """Returns {stage name: milliseconds} of one forward (synchronises the stream)."""
+    L = lib()
+    n = L.rom_num_stages()
+    ms = (ctypes.c_float * n)()
+    rc = L.rom_layer_forward_profile(ctypes.byref(cfg), ctypes.byref(weights), _ptr(x), _ptr(out), _ptr(ws), ws.numel(),
+                                     _stream(stream), ms, n)
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_layer_forward_profile")
+    return dict(zip(stage_names(), [float(v) for v in ms]))

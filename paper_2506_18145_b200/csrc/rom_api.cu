@@ -161,8 +161,18 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
   return ROM_OK;
 }
 
-int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
-                      float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream) {
+}  // extern "C"
+
+namespace rom {
+namespace {
+
+constexpr int kNumStages = 9;
+const char* const kStageNames[kNumStages] = {"route", "gather", "in_proj", "conv", "x_proj", "dt_proj", "scan", "out_proj", "combine"};
+
+// ev == nullptr: plain launch sequence.  Otherwise ev[0] is recorded before the first stage and
+// ev[i+1] after stage i (kNumStages + 1 events).
+int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
+                       float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream, cudaEvent_t* ev) {
   int rc = check_config(cfg, 0);
   if (rc != ROM_OK) return rc;
   if (!w || !x || !out || !ws) return ROM_ERR_INVALID_ARG;
@@ -186,10 +196,18 @@ int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x
   int32_t* row_of_assign = reinterpret_cast<int32_t*>(W + lay.row_of_assign);
   float* gates = gates_out ? gates_out : reinterpret_cast<float*>(W + lay.gates);
 
+  int stage = 0;
+#define ROM_STAGE_DONE()                                       \
+  do {                                                         \
+    if (ev) ROM_CUDA(cudaEventRecord(ev[++stage], st));        \
+  } while (0)
+  if (ev) ROM_CUDA(cudaEventRecord(ev[0], st));
   ROM_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t) * kStatusInts, st));
   // S1 + S2: router, top-K, permutation tables
   ROM_CUDA(launch_route(c, x, w->W_r, w->b_r, topk_idx_out, gates, counts_out, nullptr, nullptr, nullptr, W, lay, st));
+  ROM_STAGE_DONE();
   ROM_CUDA(launch_gather_rows(c, x, W, lay, st));
+  ROM_STAGE_DONE();
 
   auto gemm = [&](const void* A_, int lda, const void* B_, int ldb, int n_experts, int64_t bstride, int M_max, int Nn, int Kd,
                   const int32_t* te, const int32_t* nmt, const Epilogue& ep) -> cudaError_t {
@@ -200,25 +218,64 @@ int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x
   // S3: grouped [Conv Proj | Gate Proj]
   Epilogue e_in{EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, 0, 0};
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
+  ROM_STAGE_DONE();
   // S4: un-permute + sum over selected experts + conv + SiLU
   ROM_CUDA(launch_conv(c, W + lay.XZp, row_of_assign, w->w_conv, w->b_conv, W + lay.U, st));
+  ROM_STAGE_DONE();
   // S5: x Proj -> delta_r | B | C
   Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N};
   ROM_CUDA(gemm(W + lay.U, De, w->W_x, De, 1, 0, T, R + 2 * N, De, nullptr, nullptr, e_x));
+  ROM_STAGE_DONE();
   // S6: dt Proj + softplus
   Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0};
   ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
+  ROM_STAGE_DONE();
   // S7 + S8 + S9: scan, gate, re-permute
   const char* zbase = W + lay.XZp + (size_t)De * lay.esz;
   ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
                        reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, 2 * De, nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, st));
+  ROM_STAGE_DONE();
   // S10: grouped Out Proj
   Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0};
   ROM_CUDA(gemm(W + lay.Ygp, De, w->W_out, De, c.E, (int64_t)Dm * De, (int)lay.rows_max, Dm, De, tile_expert, num_m_tiles, e_out));
+  ROM_STAGE_DONE();
   // S11: gate-weighted combine
   ROM_CUDA(launch_combine(c, W + lay.Op, row_of_assign, gates, out, st));
+  ROM_STAGE_DONE();
+#undef ROM_STAGE_DONE
   return ROM_OK;
 }
+
+}  // namespace
+}  // namespace rom
+
+extern "C" {
+
+int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
+                      float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream) {
+  return layer_forward_impl(cfg, w, x, out, topk_idx_out, gates_out, counts_out, ws, ws_bytes, stream, nullptr);
+}
+
+int rom_layer_forward_profile(const rom_config* cfg, const rom_weights* w, const void* x, void* out, void* ws, size_t ws_bytes,
+                              void* stream, float* stage_ms, int n_stage_ms) {
+  if (!stage_ms || n_stage_ms < kNumStages) return ROM_ERR_INVALID_ARG;
+  cudaEvent_t ev[kNumStages + 1];
+  int made = 0;
+  int rc = ROM_OK;
+  for (; made <= kNumStages; ++made)
+    if (cudaEventCreate(&ev[made]) != cudaSuccess) { rc = ROM_ERR_CUDA; break; }
+  if (rc == ROM_OK) rc = layer_forward_impl(cfg, w, x, out, nullptr, nullptr, nullptr, ws, ws_bytes, stream, ev);
+  if (rc == ROM_OK && cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) rc = ROM_ERR_CUDA;
+  if (rc == ROM_OK)
+    for (int i = 0; i < kNumStages; ++i)
+      if (cudaEventElapsedTime(&stage_ms[i], ev[i], ev[i + 1]) != cudaSuccess) rc = ROM_ERR_CUDA;
+  for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
+  return rc;
+}
+
+int rom_num_stages(void) { return kNumStages; }
+
+const char* rom_stage_name(int i) { return (i >= 0 && i < kNumStages) ? kStageNames[i] : ""; }
 
 int rom_get_status(void* ws, void* stream, int32_t* host_code) {
   if (!ws || !host_code) return ROM_ERR_INVALID_ARG;
