@@ -42,7 +42,8 @@ typedef enum {
   ROM_ERR_WORKSPACE = -3,      /* ws_bytes smaller than rom_workspace_size                        */
   ROM_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (launch, tensor-map encode)   */
   ROM_ERR_ARCH = -5,           /* the current device is not sm_100                                */
-  ROM_ERR_DEVICE_TIMEOUT = -6  /* a bounded device-side wait expired (reported by rom_get_status) */
+  ROM_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired (reported by rom_get_status) */
+  ROM_ERR_STATIC_SCRATCH = -7  /* the problem does not fit the built-in scratch of rom_route_noalloc */
 } rom_status;
 
 typedef struct {
@@ -94,6 +95,31 @@ ROM_API int rom_workspace_size(const rom_config *cfg, size_t *bytes);
 ROM_API int rom_route(const rom_config *cfg, const void *x, const void *W_r, const float *b_r,
               int32_t *topk_idx, float *gates, int32_t *counts, int32_t *offsets,
               int32_t *perm, int32_t *inv_perm, void *ws, size_t ws_bytes, void *stream);
+
+/* rom_route for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a deployment variant of the routing step above, with identical results.)
+ *
+ * Who needs it: a host that gives the library a fixed set of buffers and forbids cudaMalloc while
+ * it runs -- a serving process whose memory pool belongs to another component, an allocator that
+ * is locked after start-up, a latency-critical loop that cannot absorb an allocation's cost or its
+ * failure.  Such a caller cannot provide the workspace rom_route asks for, so this entry point keeps
+ * its scratch (about 2 MiB at the largest supported size) in a fixed 3 MiB array inside the library's
+ * device image.  Every GPU that loads the library holds that array until the process exits.
+ *
+ * The caller passes inputs and outputs only; arguments, outputs and their meaning are those of
+ * rom_route.  Limits: B*L <= 65536 tokens and B*L*K <= 131072 assignments (E <= 64, K <= 8 as
+ * elsewhere); anything larger returns ROM_ERR_STATIC_SCRATCH and launches nothing -- use rom_route
+ * with a caller-owned workspace instead.  The call itself allocates nothing, on the host or device.
+ *
+ * The first call on each GPU looks up the array's device address (once per device, with that
+ * device current); make that first call before starting any stream capture.
+ * All calls on one GPU share the array, and it keeps the previous call's contents.  Each call
+ * rewrites what it reads and clears, on `stream`, the one table that must start cleared, so
+ * back-to-back calls on one stream are safe; calls that overlap on the same GPU (other streams or
+ * host threads) race on the scratch and must be serialised by the caller.                          */
+ROM_API int rom_route_noalloc(const rom_config *cfg, const void *x, const void *W_r, const float *b_r,
+                      int32_t *topk_idx, float *gates, int32_t *counts, int32_t *offsets,
+                      int32_t *perm, int32_t *inv_perm, void *stream);
 
 /* Selective scan (Section 3.1, linear recurrence h_t = A-bar h_{t-1} + B-bar U_t, Y_t = C h_t) with
  * A-bar = exp(Delta A), B-bar per disc_mode, optional skip D*U and optional gate y *= SiLU(z)

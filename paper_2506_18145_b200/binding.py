@@ -21,7 +21,7 @@ ROM_OK = 0
 
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
-           "rom_num_stages", "rom_stage_name")
+           "rom_num_stages", "rom_stage_name", "rom_route_noalloc")
 
 
 class RomConfig(ctypes.Structure):
@@ -56,6 +56,7 @@ def lib() -> ctypes.CDLL:
         cfgp = ctypes.POINTER(RomConfig)
         L.rom_workspace_size.argtypes = [cfgp, szp]
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
+        L.rom_route_noalloc.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
         L.rom_scan.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_layer_forward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, i32p, vp, i32p, vp, ctypes.c_size_t, vp]
         L.rom_workspace_find.argtypes = [cfgp, ctypes.c_char_p, szp, szp]
@@ -129,6 +130,16 @@ def rom_route(cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm
                          _ptr(offsets), _ptr(perm), _ptr(inv_perm), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_route")
+    return rc
+
+
+def rom_route_noalloc(cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm, stream=None, check=True) -> int:
+    """rom_route without a workspace argument: the scratch is a fixed array inside the library
+    (limits and sharing rules are stated beside the declaration in include/rom.h)."""
+    rc = lib().rom_route_noalloc(ctypes.byref(cfg), _ptr(x), _ptr(W_r), _ptr(b_r), _ptr(topk_idx), _ptr(gates), _ptr(counts),
+                                 _ptr(offsets), _ptr(perm), _ptr(inv_perm), _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_route_noalloc")
     return rc
 
 

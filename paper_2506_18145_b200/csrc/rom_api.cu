@@ -297,6 +297,7 @@ const char* rom_status_string(int code) {
     case ROM_ERR_CUDA: return "CUDA call failed";
     case ROM_ERR_ARCH: return "device is not sm_100";
     case ROM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case ROM_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch of rom_route_noalloc";
     default: return "unknown status";
   }
 }
