@@ -159,6 +159,53 @@ def run_reference(args, s):
     print(json.dumps(line), flush=True)
 
 
+def run_stage(args, s):
+    """One entry point alone (rom_scan or rom_route) on cuda:0 at the workload's shape, CUDA-event timed."""
+    from paper_2506_18145_b200 import binding as rb
+    rb.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    cfg = rb.config_from_shape(s)
+    if args.stage == "scan":
+        q = synth.make_scan_inputs(s.B, s.L, s.d_inner, s.d_state, s.dtype, s.seed_base + 500)
+        d = {k: (None if v is None else v.to(dev)) for k, v in q.items()}
+        y = torch.empty_like(d["u"])
+        call = lambda: rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], None, y, None)
+        esz = 2 if s.dtype == "bf16" else 4
+        nbytes = s.T * (4 * s.d_inner * esz + 8 * s.d_state)        # u, Delta, z, y at storage width; B, C fp32
+        extra = {"exps": s.T * s.d_inner * s.d_state}
+    else:
+        p = synth.make_inputs(s.replace(d_inner=64, dt_rank=16))
+        x, W_r = p["x"].to(dev), p["W_r"].to(dev)
+        b_r = None if p["b_r"] is None else p["b_r"].to(dev)
+        ws = rb.alloc_workspace(cfg, dev)
+        idx = torch.empty((s.T, s.K), dtype=torch.int32, device=dev)
+        gates = torch.empty((s.T, s.K), dtype=torch.float32, device=dev)
+        call = lambda: rb.rom_route(cfg, x, W_r, b_r, idx, gates, None, None, None, None, ws)
+        nbytes = s.T * s.d_model * x.element_size() + 16 * s.T * s.K
+        extra = {}
+    for _ in range(max(args.warmup, 3)):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    line = {"stage": args.stage, "workload": s.name, "ms": ms, "algorithmic_bytes": nbytes,
+            "achieved_gbs": nbytes / ms / 1e6, "hbm_peak_gbs": peaks["hbm_gbs"], "frac": nbytes / ms / 1e6 / peaks["hbm_gbs"],
+            "peak_source": peaks["source"]}
+    if "exps" in extra:
+        line["mufu_floor_ms"] = extra["exps"] / (148 * 16 * 1.965e9) * 1e3
+        line["mufu_frac"] = line["mufu_floor_ms"] / ms
+    print(json.dumps(line), flush=True)
+
+
 def workload_config(s):
     return {"workload": s.name, "B": s.B, "L": s.L, "d_model": s.d_model, "d_inner": s.d_inner, "d_state": s.d_state,
             "d_conv": s.d_conv, "dt_rank": s.dt_rank, "E": s.E, "K": s.K, "storage": s.dtype,
@@ -174,12 +221,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="run the projections on the fp32-FMA bisecting path")
+    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route"],
+                    help="layer: the whole forward (the benchmark); scan / route: that entry point alone, timed in isolation "
+                         "at the workload's shape (kernel studies and ncu captures; prints a short JSON line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     s = synth.CONFIGS[args.config]
 
     if args.impl == "reference":
         run_reference(args, s)
+        return
+    if args.stage != "layer":
+        run_stage(args, s)
         return
 
     from paper_2506_18145_b200 import binding as rb

@@ -35,6 +35,7 @@ WsLayout make_layout(const rom_config& c) {
   l.x_perm = take(l.esz * (size_t)l.rows_max * c.d_model);
   l.XZp = take(l.esz * (size_t)l.rows_max * 2 * c.d_inner);
   l.U = take(l.esz * (size_t)l.T * c.d_inner);
+  l.Zs = take(c.K > 1 ? l.esz * (size_t)l.T * c.d_inner : 0);   // gate rows summed over the K slots
   l.delta_r = take(l.esz * (size_t)l.T * R);
   l.Bm = take(sizeof(float) * (size_t)l.T * N);
   l.Cm = take(sizeof(float) * (size_t)l.T * N);
@@ -157,7 +158,7 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
   if ((rc = check_device()) != ROM_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   LaunchCounter::count = 0;
-  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, h0, y, h_last, nullptr, 1, st));
+  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, st));
   return ROM_OK;
 }
 
@@ -220,7 +221,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
   ROM_STAGE_DONE();
   // S4: un-permute + sum over selected experts + conv + SiLU
-  ROM_CUDA(launch_conv(c, W + lay.XZp, row_of_assign, w->w_conv, w->b_conv, W + lay.U, st));
+  ROM_CUDA(launch_conv(c, W + lay.XZp, row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
   ROM_STAGE_DONE();
   // S5: x Proj -> delta_r | B | C
   Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N};
@@ -231,9 +232,11 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
   ROM_STAGE_DONE();
   // S7 + S8 + S9: scan, gate, re-permute
-  const char* zbase = W + lay.XZp + (size_t)De * lay.esz;
+  // K = 1: the gate row of a token is its Gate Proj row in expert order; K > 1: the summed rows from S4
+  const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;
   ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
-                       reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, 2 * De, nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, st));
+                       reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, c.K == 1 ? row_of_assign : nullptr,
+                       nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, st));
   ROM_STAGE_DONE();
   // S10: grouped Out Proj
   Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0};

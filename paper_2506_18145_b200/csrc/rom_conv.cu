@@ -40,31 +40,52 @@ __device__ __forceinline__ void store_vec(float* p, const float (&v)[4]) {
   *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
 }
 
-// H row of token t (global token index) = sum over its K slots of the first D_e columns of XZp.
-template <typename T, int V>
-__device__ __forceinline__ void load_h(const T* XZp, int ld, const int32_t* row_of_assign, int K, int t, int c0, float (&h)[V]) {
+// Sum over the K slots of a token of one 16-byte vector of a [rows, ld] matrix (fp32 accumulation).
+template <typename T, int V, int KT>
+__device__ __forceinline__ void load_sum(const T* M, int ld, const int32_t* row_of_assign, int K, size_t t, int c0, float (&h)[V]) {
+  if constexpr (KT == 1) {
+    load_vec(M + (size_t)__ldg(row_of_assign + t) * ld + c0, h);
+  } else {
+    const int kk = KT > 0 ? KT : K;
 #pragma unroll
-  for (int i = 0; i < V; ++i) h[i] = 0.0f;
-  for (int k = 0; k < K; ++k) {
-    const int row = __ldg(row_of_assign + (size_t)t * K + k);
-    float v[V];
-    load_vec(XZp + (size_t)row * ld + c0, v);
+    for (int i = 0; i < V; ++i) h[i] = 0.0f;
 #pragma unroll
-    for (int i = 0; i < V; ++i) h[i] += v[i];
+    for (int k = 0; k < kk; ++k) {
+      float v[V];
+      load_vec(M + (size_t)__ldg(row_of_assign + t * kk + k) * ld + c0, v);
+#pragma unroll
+      for (int i = 0; i < V; ++i) h[i] += v[i];
+    }
   }
 }
 
-template <typename T>
+// One thread: one 16-byte vector of channels, TCH consecutive time steps of one sequence.  All rows it
+// needs (TCH + 3 of H, TCH of Z when Zs != nullptr) are loaded before anything is consumed, so the
+// memory system sees TCH + 3 independent requests per thread.  KT > 0 fixes K at compile time.
+constexpr int TCH = 8;
+
+template <typename T, int KT>
 __global__ void __launch_bounds__(128)
 conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_assign, const T* __restrict__ w_conv,
-                 const float* __restrict__ b_conv, T* __restrict__ U, int L, int De, int K, int dconv, int tchunk) {
+                 const float* __restrict__ b_conv, T* __restrict__ U, T* __restrict__ Zs, int L, int De, int K, int dconv) {
   constexpr int V = Vec<T>::N;
   const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * V;
   if (c0 >= De) return;
   const int b = blockIdx.z;
-  const int tb = blockIdx.y * tchunk;
-  const int te = min(L, tb + tchunk);
+  const int tb = blockIdx.y * TCH;
   const int ld = 2 * De;
+  const size_t tok0 = (size_t)b * L;
+
+  float hrow[TCH + 3][V];                 // rows tb-3 .. tb+TCH-1
+#pragma unroll
+  for (int r = 0; r < TCH + 3; ++r) {
+    const int t = tb - 3 + r;
+    if (t >= 0 && t < L) load_sum<T, V, KT>(XZp, ld, row_of_assign, K, tok0 + t, c0, hrow[r]);
+    else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) hrow[r][i] = 0.0f;
+    }
+  }
   // taps right-aligned into 4 slots: slot 3 multiplies the current token
   float w[4][V];
 #pragma unroll
@@ -79,37 +100,33 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
   float bias[V];
 #pragma unroll
   for (int i = 0; i < V; ++i) bias[i] = b_conv ? b_conv[c0 + i] : 0.0f;
-  float h1[V], h2[V], h3[V];     // rows t-1, t-2, t-3
-  const size_t tok0 = (size_t)b * L;
-  if (tb - 1 >= 0) load_h<T, V>(XZp, ld, row_of_assign, K, (int)(tok0 + tb - 1), c0, h1);
-  else {
+
 #pragma unroll
-    for (int i = 0; i < V; ++i) h1[i] = 0.0f;
-  }
-  if (tb - 2 >= 0) load_h<T, V>(XZp, ld, row_of_assign, K, (int)(tok0 + tb - 2), c0, h2);
-  else {
-#pragma unroll
-    for (int i = 0; i < V; ++i) h2[i] = 0.0f;
-  }
-  if (tb - 3 >= 0) load_h<T, V>(XZp, ld, row_of_assign, K, (int)(tok0 + tb - 3), c0, h3);
-  else {
-#pragma unroll
-    for (int i = 0; i < V; ++i) h3[i] = 0.0f;
-  }
-  for (int t = tb; t < te; ++t) {
-    float h0[V], u[V];
-    load_h<T, V>(XZp, ld, row_of_assign, K, (int)(tok0 + t), c0, h0);
+  for (int r = 0; r < TCH; ++r) {
+    const int t = tb + r;
+    if (t >= L) break;
+    float u[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) {
       float pre = bias[i];
-      pre = fmaf(w[0][i], h3[i], pre);
-      pre = fmaf(w[1][i], h2[i], pre);
-      pre = fmaf(w[2][i], h1[i], pre);
-      pre = fmaf(w[3][i], h0[i], pre);
+      pre = fmaf(w[0][i], hrow[r][i], pre);
+      pre = fmaf(w[1][i], hrow[r + 1][i], pre);
+      pre = fmaf(w[2][i], hrow[r + 2][i], pre);
+      pre = fmaf(w[3][i], hrow[r + 3][i], pre);
       u[i] = silu_f(pre);
-      h3[i] = h2[i]; h2[i] = h1[i]; h1[i] = h0[i];
     }
     store_vec(U + (tok0 + t) * De + c0, u);
+  }
+  if (Zs != nullptr) {
+    // gate pre-activation summed over the selected experts (indicator only), one row per token
+#pragma unroll
+    for (int r = 0; r < TCH; ++r) {
+      const int t = tb + r;
+      if (t >= L) break;
+      float zsum[V];
+      load_sum<T, V, KT>(XZp + De, ld, row_of_assign, K, tok0 + t, c0, zsum);
+      store_vec(Zs + (tok0 + t) * De + c0, zsum);
+    }
   }
 }
 
@@ -140,21 +157,28 @@ combine_kernel(const T* __restrict__ Op, const int32_t* __restrict__ row_of_assi
 
 }  // namespace
 
-cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
-                        const float* b_conv, void* U, cudaStream_t st) {
-  const int tchunk = 64;
-  const bool bf = c.dtype == ROM_BF16;
-  const int V = bf ? 8 : 4;
+template <typename T>
+cudaError_t launch_conv_t(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
+                          const float* b_conv, void* U, void* Zs, cudaStream_t st) {
+  constexpr int V = Vec<T>::N;
   const int threads = 128;
-  dim3 grid((c.d_inner / V + threads - 1) / threads, (c.L + tchunk - 1) / tchunk, c.B);
-  if (bf)
-    conv_silu_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((const __nv_bfloat16*)XZp, row_of_assign, (const __nv_bfloat16*)w_conv,
-                                                             b_conv, (__nv_bfloat16*)U, c.L, c.d_inner, c.K, c.d_conv, tchunk);
-  else
-    conv_silu_kernel<float><<<grid, threads, 0, st>>>((const float*)XZp, row_of_assign, (const float*)w_conv, b_conv, (float*)U,
-                                                     c.L, c.d_inner, c.K, c.d_conv, tchunk);
+  dim3 grid((c.d_inner / V + threads - 1) / threads, (c.L + TCH - 1) / TCH, c.B);
+  auto args = [&](auto kern) {
+    kern<<<grid, threads, 0, st>>>((const T*)XZp, row_of_assign, (const T*)w_conv, b_conv, (T*)U, (T*)Zs, c.L, c.d_inner, c.K, c.d_conv);
+  };
+  if (c.K == 1) args(conv_silu_kernel<T, 1>);
+  else if (c.K == 2) args(conv_silu_kernel<T, 2>);
+  else args(conv_silu_kernel<T, 0>);
   count_launch();
   return cudaGetLastError();
+}
+
+// Zs: [T, d_inner] sum over the K slots of the Gate Proj rows, or nullptr (not produced).
+cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
+                        const float* b_conv, void* U, void* Zs, cudaStream_t st) {
+  if (c.B > 65535 || (c.L + TCH - 1) / TCH > 65535) return cudaErrorInvalidConfiguration;
+  return c.dtype == ROM_BF16 ? launch_conv_t<__nv_bfloat16>(c, XZp, row_of_assign, w_conv, b_conv, U, Zs, st)
+                             : launch_conv_t<float>(c, XZp, row_of_assign, w_conv, b_conv, U, Zs, st);
 }
 
 cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,

@@ -25,7 +25,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct WsLayout {
   size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts;
   size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
-  size_t x_perm, XZp, U, delta_r, Bm, Cm, Delta, Ygp, Op;
+  size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op;
   size_t total;
   int64_t T, A, rows_max, max_m_tiles, n_chunks;
   size_t esz;
@@ -69,14 +69,14 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
                            const Epilogue& epi, int32_t* status, cudaStream_t st);
 
 cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
-                        const float* b_conv, void* U, cudaStream_t st);
+                        const float* b_conv, void* U, void* Zs, cudaStream_t st);
 
-// Scan.  row_map == nullptr: y is [T, d_inner] and z is [T, ldz]; otherwise y row of (t, k) is
-// row_map[t*K + k] (K rows written per token) and z is read from row row_map[t*K + k] of a
-// [rows, ldz] matrix and summed over k.
+// Scan.  z is a [rows, ldz] matrix; the gate row of token t is z_row[t] (z_row == nullptr: row t).
+// y_rows == nullptr: y is [T, d_inner]; otherwise the output row of token t is written K times, to rows
+// y_rows[t*K + k].
 cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
-                        const float* Cm, const float* D, const void* z, int ldz, const float* h0, void* y,
-                        float* h_last, const int32_t* row_map, int K, cudaStream_t st);
+                        const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
+                        void* y, float* h_last, const int32_t* y_rows, int K, cudaStream_t st);
 
 cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,
                            void* out, cudaStream_t st);

@@ -2,16 +2,32 @@
 // fused with the output gate y * SiLU(z) and with the re-permutation of the gated rows into expert
 // order (the routing decision of the Gate/Conv projections is reused for Out Proj, Section 4.2).
 //
-// State and arithmetic are fp32.  One thread owns one channel and keeps its d_state = 16 states in
-// registers; consecutive lanes own consecutive channels, so every load and store of u, Delta, z, y
-// is coalesced.  B_t / C_t are staged through shared memory per block of time steps.
+// State and arithmetic are fp32.  The recurrence is sequential in t, so the parallelism is
+// (sequence, channel, state).  One thread owns NS of the 16 states of NC adjacent channels
+// (registers, packed pairs); the S = 16/NS lanes of a channel group are adjacent.  Per state and step
+// the work is one exponential on the special-function unit (16 per clock per SM: the binding limit),
+// about six fp32 multiply/FMA lanes, and the shared-memory words for (Delta, u) and (B, C).  The
+// launcher picks the largest work per thread that still fills the GPU (small NS only for a single
+// long sequence).
+//
+// A block of 256 threads owns CH = NC*256/S channels of one sequence and walks the sequence in tiles
+// of TS = 2048/CH steps, so every thread also owns one (row, 8 channels) piece of each tile: it
+// fetches that piece of tile i+1 (Delta, u, z) from global memory into registers -- raw,
+// unconverted, so nothing waits on the loads -- while tile i is computed from shared memory, then
+// converts and stores it to the other shared buffer.  The scan proper leaves sum_n C h in shared
+// memory; the skip term, the gate, the rounding and the 16-byte row stores are done by the thread
+// that loaded that piece, which still holds u and z in registers.  One __syncthreads per tile.  The
+// per-channel operands are stored duplicated, (Delta, Delta, v, v), so one 16-byte load yields both
+// packed operands; 8-channel groups are XOR-swizzled so that loader stores and compute loads are
+// both bank-conflict free.
 #include "rom_internal.cuh"
 
 namespace rom {
 namespace {
 
-constexpr int NST = 16;        // d_state
-constexpr int TS = 64;         // time steps of B/C staged per shared-memory tile
+constexpr int NST = 16;            // d_state
+constexpr int BLOCK = 256;
+constexpr int TILE_ELEMS = 2048;   // (time steps) x (channels) per tile = 8 per thread
 constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -20,93 +36,363 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
-// PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance).
-// otherwise: one MUFU ex2 per state update; expm1 taken as a - 1 (bf16 configurations).
-template <typename T, bool PRECISE>
-__global__ void __launch_bounds__(128)
-scan_kernel(const T* __restrict__ u, const float* __restrict__ delta, const float* __restrict__ A,
-            const float* __restrict__ Bm, const float* __restrict__ Cm, const float* __restrict__ D,
-            const T* __restrict__ z, int ldz, const float* __restrict__ h0, T* __restrict__ y,
-            float* __restrict__ h_last, const int32_t* __restrict__ row_map, int K, int L, int De, int disc_mode) {
-  __shared__ float Bs[TS][NST];
-  __shared__ float Cs[TS][NST];
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  const int b = blockIdx.y;
-  const bool active = c < De;
-  const int cc = active ? c : De - 1;
-
-  float a_n[NST], inv_a[NST], h[NST];
+// 8 consecutive elements of a row, kept raw (16-byte words) until consumed.
+template <typename T> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+  uint4 q;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ __forceinline__ void zero() { q = make_uint4(0, 0, 0, 0); }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-  for (int n = 0; n < NST; ++n) {
-    const float av = A[(size_t)cc * NST + n];
-    a_n[n] = PRECISE ? av : av * kLog2e;
-    inv_a[n] = 1.0f / av;
-    h[n] = h0 ? h0[((size_t)b * De + cc) * NST + n] : 0.0f;
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
   }
-  const float dskip = D ? D[cc] : 0.0f;
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8]) {
+    uint4 o;
+    uint32_t* w = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 hh = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+      w[i] = *reinterpret_cast<const uint32_t*>(&hh);
+    }
+    *reinterpret_cast<uint4*>(p) = o;
+  }
+};
+template <> struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) {
+    a = __ldg(reinterpret_cast<const float4*>(p));
+    b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+  }
+  __device__ __forceinline__ void zero() { a = make_float4(0.0f, 0.0f, 0.0f, 0.0f); b = a; }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+  static __device__ __forceinline__ void store(float* p, const float (&v)[8]) {
+    reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+};
+
+template <int NC, int NS>
+struct Geo {
+  static constexpr int S = NST / NS;                    // lanes per channel group
+  static constexpr int NP = NS / 2;                     // packed state pairs per channel per thread
+  static constexpr int CH = BLOCK / S * NC;             // channels per block
+  static constexpr int TS = TILE_ELEMS / CH;            // time steps per tile
+  static constexpr int CG = CH / 8;                     // 8-channel groups (= loader threads) per row
+  static constexpr int SLOT = 32 + 32 / S;              // words per time slot of the partial-sum strip (padded)
+  static constexpr int STRIP = S > 4 ? S * SLOT : 0;    // words per warp (only the 8-lane split uses the strip)
+  static constexpr int YP = CH + (S > 4 ? 4 : 0);       // row pitch (words) of the staged sums
+  static constexpr int NBC = TS * 32 / BLOCK;           // B/C words fetched per thread per tile
+  static_assert(NS % 2 == 0 && S >= 1 && S <= 8 && TS % S == 0 && CG * TS == BLOCK && (NC == 1 || S <= 4), "unsupported split");
+};
+
+// position of channel c inside its tile row: the 8 channels of a group are permuted by the group index
+__device__ __forceinline__ int swz(int c) { return (c & ~7) | ((c ^ (c >> 3)) & 7); }
+
+// Shared-memory image of one input tile.
+template <int NC, int NS>
+struct Tile {
+  float4 dv[Geo<NC, NS>::TS][Geo<NC, NS>::CH];   // (Delta, Delta, v, v) at [t][swz(c)]: v = u (zero-order hold) or Delta*u
+  float4 bc[Geo<NC, NS>::TS][NST / 2];           // (B_n, B_n+1, C_n, C_n+1) per state pair
+};
+
+struct ScanArgs {
+  const void* u; const float* delta; const float* A; const float* Bm; const float* Cm; const float* D;
+  const void* z; int ldz; const int32_t* z_row; const float* h0; void* y; float* h_last; const int32_t* y_rows;
+  int K, L, De;
+};
+
+// PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance); otherwise one ex2.approx per
+// state update (bf16 configurations, 2e-2 tolerance).
+// ZOH: zero-order-hold B-bar (disc_mode 0); otherwise B-bar = Delta B.
+template <typename T, int NC, int NS, bool PRECISE, bool ZOH>
+__global__ void __launch_bounds__(BLOCK, NS >= 8 ? 2 : 1)
+scan_kernel(const ScanArgs p) {
+  using G = Geo<NC, NS>;
+  using TileT = Tile<NC, NS>;
+  constexpr int S = G::S, NP = G::NP, CH = G::CH, TS = G::TS, YP = G::YP;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  TileT* tiles = reinterpret_cast<TileT*>(smem_raw);                                        // [2]
+  float* ysum = reinterpret_cast<float*>(smem_raw + 2 * sizeof(TileT));                     // [2][TS][YP]
+  float* ps_all = ysum + 2 * TS * YP;                                                       // [8 warps][STRIP]
+
+  const T* __restrict__ u = static_cast<const T*>(p.u);
+  const T* __restrict__ z = static_cast<const T*>(p.z);
+  T* __restrict__ y = static_cast<T*>(p.y);
+  const int L = p.L, De = p.De, K = p.K;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.y;
+  const int c_base = blockIdx.x * CH;
   const size_t tok0 = (size_t)b * L;
 
-  for (int t0 = 0; t0 < L; t0 += TS) {
-    const int nt = min(TS, L - t0);
-    __syncthreads();
-    for (int i = threadIdx.x; i < nt * NST; i += blockDim.x) {
-      (&Bs[0][0])[i] = Bm[(tok0 + t0) * NST + i];
-      (&Cs[0][0])[i] = Cm[(tok0 + t0) * NST + i];
-    }
-    __syncthreads();
-    for (int tt = 0; tt < nt; ++tt) {
-      const size_t tok = tok0 + t0 + tt;
-      const float dl = delta[tok * De + cc];
-      const float uu = to_f32(u[tok * De + cc]);
-      float acc = 0.0f;
+  // ---- compute role: NC adjacent channels from block-local channel cl, states [g*NS, g*NS+NS)
+  const int cl = (tid / S) * NC, g = tid % S;
+  float2 a2[NC][NP], kin[NC][NP], h[NC][NP];
+  int cl_sw[NC];
 #pragma unroll
-      for (int n = 0; n < NST; ++n) {
-        float a, bbar;
-        if (PRECISE) {
-          const float dA = dl * a_n[n];
-          a = expf(dA);
-          bbar = (disc_mode == 0) ? expm1f(dA) * inv_a[n] * Bs[tt][n] : dl * Bs[tt][n];
-        } else {
-          a = ex2_approx(dl * a_n[n]);
-          bbar = (disc_mode == 0) ? (a - 1.0f) * inv_a[n] * Bs[tt][n] : dl * Bs[tt][n];
-        }
-        h[n] = fmaf(a, h[n], bbar * uu);
-        acc = fmaf(Cs[tt][n], h[n], acc);
+  for (int i = 0; i < NC; ++i) {
+    const int c = min(c_base + cl + i, De - 1);
+    cl_sw[i] = swz(cl + i);
+#pragma unroll
+    for (int q = 0; q < NP; ++q) {
+      const int n = g * NS + 2 * q;
+      const float a0 = p.A[(size_t)c * NST + n], a1 = p.A[(size_t)c * NST + n + 1];
+      a2[i][q] = PRECISE ? make_float2(a0, a1) : make_float2(a0 * kLog2e, a1 * kLog2e);
+      kin[i][q] = make_float2(-1.0f / a0, -1.0f / a1);
+      h[i][q] = p.h0 ? make_float2(p.h0[((size_t)b * De + c) * NST + n], p.h0[((size_t)b * De + c) * NST + n + 1])
+                     : make_float2(0.0f, 0.0f);
+    }
+  }
+  float* ps = ps_all + warp * G::STRIP;
+
+  // ---- loader / finisher role: row lr of every tile, channels [lc, lc + 8)
+  const int lr = tid / G::CG, lc = (tid % G::CG) * 8;
+  const bool lc_ok = c_base + lc < De;
+  const int lc_eff = lc_ok ? c_base + lc : 0;
+  float dsk[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) dsk[i] = p.D ? p.D[lc_eff + i] : 0.0f;
+  // running pointers to this thread's piece of the next tile to fetch
+  const float* dptr = p.delta + (tok0 + lr) * De + lc_eff;
+  const T* uptr = u + (tok0 + lr) * De + lc_eff;
+  const size_t row_step = (size_t)TS * De;
+  // B/C: word i of this thread is element (r = warp + 8 i, j = lane) of the [TS][32] tile (B | C)
+  const float* bcptr = (lane < NST ? p.Bm : p.Cm) + (tok0 + warp) * NST + (lane & 15);
+  const int bc_dst = ((lane & 15) >> 1) * 4 + ((lane >> 4) << 1) + (lane & 1);
+
+  Raw8<float> pre_d;
+  Raw8<T> pre_u, pre_z, cur_u, cur_z;
+  float pre_bc[G::NBC];
+
+  auto fetch = [&](int t0) {        // global -> registers, no conversion
+    const int t = t0 + lr;
+    pre_d.zero(); pre_u.zero(); pre_z.zero();
+    if (lc_ok && t < L) {
+      pre_d.load(dptr);
+      pre_u.load(uptr);
+      if (z) {
+        const size_t zrow = p.z_row ? (size_t)__ldg(p.z_row + tok0 + t) : tok0 + t;
+        pre_z.load(z + zrow * p.ldz + lc_eff);
       }
-      acc = fmaf(dskip, uu, acc);
-      if (row_map == nullptr) {
-        if (z) acc *= silu_f(to_f32(z[tok * ldz + cc]));
-        if (active) y[tok * De + cc] = from_f32<T>(acc);
+    }
+    dptr += row_step; uptr += row_step;
+#pragma unroll
+    for (int i = 0; i < G::NBC; ++i) pre_bc[i] = (t0 + warp + 8 * i < L) ? __ldg(bcptr + i * 8 * NST) : 0.0f;
+    bcptr += TS * NST;
+  };
+  auto stash = [&](TileT& tl) {     // registers -> shared, converting
+    float d[8], uu[8];
+    pre_d.get(d); pre_u.get(uu);
+    float4* row = &tl.dv[lr][lc];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float v = ZOH ? uu[i] : d[i] * uu[i];
+      row[i ^ ((lc >> 3) & 7)] = make_float4(d[i], d[i], v, v);
+    }
+#pragma unroll
+    for (int i = 0; i < G::NBC; ++i) reinterpret_cast<float*>(&tl.bc[warp + 8 * i][0])[bc_dst] = pre_bc[i];
+  };
+  // y = (sum_n C h + D u) * SiLU(z), rounded, written to the K output rows of the token
+  auto flush = [&](int t0, const float* ys) {
+    const int t = t0 + lr;
+    if (!lc_ok || t >= L) return;
+    float uu[8], o[8];
+    cur_u.get(uu);
+    const float4 s0 = *reinterpret_cast<const float4*>(ys + lr * YP + lc), s1 = *reinterpret_cast<const float4*>(ys + lr * YP + lc + 4);
+    const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = fmaf(dsk[i], uu[i], sv[i]);
+    if (z) {
+      float zz[8];
+      cur_z.get(zz);
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        o[i] *= PRECISE ? zz[i] / (1.0f + expf(-zz[i])) : __fdividef(zz[i], 1.0f + __expf(-zz[i]));
+    }
+    const size_t tok = tok0 + t;
+    if (p.y_rows == nullptr) {
+      Raw8<T>::store(y + tok * De + lc_eff, o);
+    } else {
+      for (int kk = 0; kk < K; ++kk) Raw8<T>::store(y + (size_t)__ldg(p.y_rows + tok * K + kk) * De + lc_eff, o);
+    }
+  };
+
+  fetch(0);
+  stash(tiles[0]);
+  cur_u = pre_u; cur_z = pre_z;
+  __syncthreads();
+
+  int buf = 0;
+  for (int t0 = 0; t0 < L; t0 += TS, buf ^= 1) {
+    const bool more = t0 + TS < L;
+    if (more) fetch(t0 + TS);
+    const TileT& tl = tiles[buf];
+    float* ys = ysum + buf * TS * YP;
+
+    // Plain loop over the steps of the tile: loads, exponentials and the recurrence of one step in
+    // program order, unrolled a few steps so the scheduler can overlap them.  The restrict-qualified
+    // views tell the compiler that the stores of the sums never alias the tile it reads.
+    const float4* __restrict__ dvp = &tl.dv[0][0];
+    const float4* __restrict__ bcp = &tl.bc[0][g * NP];
+    float* __restrict__ ysp = ys + cl;
+    float* __restrict__ psp = ps;
+    constexpr int UF = S > 4 ? S : (NC * NS >= 16 ? 2 : 4);
+#pragma unroll UF
+    for (int tt = 0; tt < TS; ++tt) {
+      float4 bc[NP];
+#pragma unroll
+      for (int q = 0; q < NP; ++q) bc[q] = bcp[tt * (NST / 2) + q];
+      float part[NC];
+#pragma unroll
+      for (int i = 0; i < NC; ++i) {
+        const float4 dv = dvp[tt * CH + cl_sw[i]];
+        const float2 dl2 = make_float2(dv.x, dv.y), vv2 = make_float2(dv.z, dv.w);
+        float2 acc0 = make_float2(0.0f, 0.0f), acc1 = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int q = 0; q < NP; ++q) {
+          const float2 Bv = make_float2(bc[q].x, bc[q].y), Cv = make_float2(bc[q].z, bc[q].w);
+          if (PRECISE) {
+            const float dA0 = dl2.x * a2[i][q].x, dA1 = dl2.x * a2[i][q].y;
+            // B-bar u: zero-order hold expm1(dA)/A * B * u, or (Delta u) * B
+            const float w0 = ZOH ? -expm1f(dA0) * kin[i][q].x * Bv.x * vv2.x : Bv.x * vv2.x;
+            const float w1 = ZOH ? -expm1f(dA1) * kin[i][q].y * Bv.y * vv2.x : Bv.y * vv2.x;
+            h[i][q].x = fmaf(expf(dA0), h[i][q].x, w0);
+            h[i][q].y = fmaf(expf(dA1), h[i][q].y, w1);
+            acc0.x = fmaf(Cv.x, h[i][q].x, acc0.x);
+            acc0.y = fmaf(Cv.y, h[i][q].y, acc0.y);
+          } else {
+            const float2 x = __fmul2_rn(dl2, a2[i][q]);
+            const float2 a = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+            if (ZOH) {
+              // zero-order hold: w = -B u / A, h <- a (h - w) + w = a h + (a - 1) B u / A
+              const float2 w = __fmul2_rn(__fmul2_rn(vv2, kin[i][q]), Bv);
+              const float2 sdiff = __ffma2_rn(w, make_float2(-1.0f, -1.0f), h[i][q]);
+              h[i][q] = __ffma2_rn(a, sdiff, w);
+            } else {
+              h[i][q] = __ffma2_rn(a, h[i][q], __fmul2_rn(vv2, Bv));      // w = (Delta u) B
+            }
+            float2& acc = (q & 1) ? acc1 : acc0;
+            acc = q < 2 ? __fmul2_rn(Cv, h[i][q]) : __ffma2_rn(Cv, h[i][q], acc);
+          }
+        }
+        if (NP > 1 && !PRECISE) acc0 = __fadd2_rn(acc0, acc1);
+        part[i] = acc0.x + acc0.y;
+      }
+      if (S == 1) {
+#pragma unroll
+        for (int i = 0; i < NC; ++i) ysp[tt * YP + i] = part[i];
+      } else if (S <= 4) {
+        // all S lanes of the channel get the sum; lane g stores the steps with tt % S == g
+#pragma unroll
+        for (int i = 0; i < NC; ++i) {
+#pragma unroll
+          for (int o = 1; o < S; o <<= 1) part[i] += __shfl_xor_sync(0xffffffffu, part[i], o);
+        }
+        if ((tt % S) == g) {
+#pragma unroll
+          for (int i = 0; i < NC; ++i) ysp[tt * YP + i] = part[i];
+        }
       } else {
-        float zs = 0.0f;
-        for (int k = 0; k < K; ++k) zs += to_f32(z[(size_t)row_map[tok * K + k] * ldz + cc]);
-        acc *= silu_f(zs);
-        if (active)
-          for (int k = 0; k < K; ++k) y[(size_t)row_map[tok * K + k] * De + cc] = from_f32<T>(acc);
+        psp[(tt % S) * G::SLOT + lane] = part[0];
+        if ((tt % S) == S - 1) {
+          __syncwarp();
+          // lane g of the channel adds up the S partial sums of time step tt - (S-1) + g
+          const float* src = psp + g * G::SLOT + (lane / S) * S;
+          float sum = 0.0f;
+#pragma unroll
+          for (int j = 0; j < S; j += 4) {
+            const float4 v4 = *reinterpret_cast<const float4*>(src + j);
+            sum += (v4.x + v4.y) + (v4.z + v4.w);
+          }
+          ysp[(tt - (S - 1) + g) * YP] = sum;
+          __syncwarp();
+        }
+      }
+    }
+
+    if (more) stash(tiles[buf ^ 1]);
+    __syncthreads();
+    flush(t0, ys);
+    if (more) { cur_u = pre_u; cur_z = pre_z; }
+  }
+
+  if (p.h_last) {
+#pragma unroll
+    for (int i = 0; i < NC; ++i) {
+      const int c = c_base + cl + i;
+      if (c >= De) continue;
+#pragma unroll
+      for (int q = 0; q < NP; ++q) {
+        const int n = g * NS + 2 * q;
+        p.h_last[((size_t)b * De + c) * NST + n] = h[i][q].x;
+        p.h_last[((size_t)b * De + c) * NST + n + 1] = h[i][q].y;
       }
     }
   }
-  if (h_last && active) {
-#pragma unroll
-    for (int n = 0; n < NST; ++n) h_last[((size_t)b * De + c) * NST + n] = h[n];
+}
+
+template <typename T, int NC, int NS, bool PRECISE, bool ZOH>
+cudaError_t launch_one(const ScanArgs& a, int B, cudaStream_t st) {
+  using G = Geo<NC, NS>;
+  const size_t smem = 2 * sizeof(Tile<NC, NS>) + (2 * (size_t)G::TS * G::YP + (BLOCK / 32) * G::STRIP) * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, NC, NS, PRECISE, ZOH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid((a.De + G::CH - 1) / G::CH, B);
+  scan_kernel<T, NC, NS, PRECISE, ZOH><<<grid, BLOCK, smem, st>>>(a);
+  return cudaGetLastError();
+}
+
+// Work per thread, NC channels x NS states, as NC * 100 + NS: the largest of 1x8, 1x4, 1x2 that still
+// gives every SM sub-partition about two warps.
+int pick_thread_shape(int B, int De, int num_sms) {
+  const long long want_warps = 2LL * 4 * num_sms;
+  const int shapes[2][2] = {{1, 8}, {1, 4}};
+  for (const auto& sh : shapes) {
+    const int ch = BLOCK / (NST / sh[1]) * sh[0];
+    const long long warps = (long long)B * ((De + ch - 1) / ch) * (BLOCK / 32);
+    if (warps >= want_warps) return sh[0] * 100 + sh[1];
+  }
+  return 102;
+}
+
+template <typename T, bool PRECISE, bool ZOH>
+cudaError_t launch_shape(int shape, const ScanArgs& a, int B, cudaStream_t st) {
+  switch (shape) {
+    case 208: return launch_one<T, 2, 8, PRECISE, ZOH>(a, B, st);
+    case 108: return launch_one<T, 1, 8, PRECISE, ZOH>(a, B, st);
+    case 104: return launch_one<T, 1, 4, PRECISE, ZOH>(a, B, st);
+    case 102: return launch_one<T, 1, 2, PRECISE, ZOH>(a, B, st);
+    default: return cudaErrorInvalidValue;
   }
 }
 
 }  // namespace
 
 cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
-                        const float* Cm, const float* D, const void* z, int ldz, const float* h0, void* y,
-                        float* h_last, const int32_t* row_map, int K, cudaStream_t st) {
-  const int threads = 64;
-  dim3 grid((c.d_inner + threads - 1) / threads, c.B);
+                        const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
+                        void* y, float* h_last, const int32_t* y_rows, int K, cudaStream_t st) {
+  static int num_sms = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+  }
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner};
+  const int shape = pick_thread_shape(c.B, c.d_inner, num_sms);
+  cudaError_t e;
   if (c.dtype == ROM_BF16)
-    scan_kernel<__nv_bfloat16, false><<<grid, threads, 0, st>>>((const __nv_bfloat16*)u, delta, A, Bm, Cm, D, (const __nv_bfloat16*)z, ldz,
-                                                               h0, (__nv_bfloat16*)y, h_last, row_map, K, c.L, c.d_inner, c.disc_mode);
+    e = c.disc_mode == 0 ? launch_shape<__nv_bfloat16, false, true>(shape, a, c.B, st) : launch_shape<__nv_bfloat16, false, false>(shape, a, c.B, st);
   else
-    scan_kernel<float, true><<<grid, threads, 0, st>>>((const float*)u, delta, A, Bm, Cm, D, (const float*)z, ldz, h0, (float*)y,
-                                                      h_last, row_map, K, c.L, c.d_inner, c.disc_mode);
+    e = c.disc_mode == 0 ? launch_shape<float, true, true>(shape, a, c.B, st) : launch_shape<float, true, false>(shape, a, c.B, st);
   count_launch();
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace rom
