@@ -113,7 +113,7 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
       pre = fmaf(w[1][i], hrow[r + 1][i], pre);
       pre = fmaf(w[2][i], hrow[r + 2][i], pre);
       pre = fmaf(w[3][i], hrow[r + 3][i], pre);
-      u[i] = silu_f(pre);
+      u[i] = sizeof(T) == 2 ? silu_fast(pre) : silu_f(pre);
     }
     store_vec(U + (tok0 + t) * De + c0, u);
   }

@@ -128,7 +128,7 @@ __device__ __forceinline__ void epi_store8(const Epilogue& ep, size_t m, int n0,
   } else {
     float o[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) o[i] = softplus_f(v[i] + (ep.bias ? __ldg(ep.bias + n0 + i) : 0.0f));
+    for (int i = 0; i < 8; ++i) o[i] = softplus_fast(v[i] + (ep.bias ? __ldg(ep.bias + n0 + i) : 0.0f));
     float* dst = reinterpret_cast<float*>(ep.C) + m * ep.ldc + n0;
     *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
     *reinterpret_cast<float4*>(dst + 4) = make_float4(o[4], o[5], o[6], o[7]);

@@ -89,6 +89,15 @@ template <> __device__ __forceinline__ float from_f32<float>(float v) { return v
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
+// Fast forms for the bf16 path (results are rounded to bf16 or feed a 2e-2 tolerance): approximate
+// reciprocal / exp2 / log2 of the special-function unit, relative error ~1e-6.
+__device__ __forceinline__ float silu_fast(float v) { return __fdividef(v, 1.0f + __expf(-v)); }
+__device__ __forceinline__ float softplus_fast(float v) {
+  // max(v,0) + log(1 + e), e = exp(-|v|) in (0, 1].  For tiny e, 1 + e loses e's low bits: use log1p(e) ~ e.
+  const float e = __expf(-fabsf(v));
+  const float l = e < 2.44140625e-4f ? e : __logf(1.0f + e);
+  return fmaxf(v, 0.0f) + l;
+}
 __device__ __forceinline__ float softplus_f(float v) {
   // max(v,0) + log1p(exp(-|v|)); log1pf keeps relative accuracy when exp(-|v|) is tiny
   return fmaxf(v, 0.0f) + log1pf(__expf(-fabsf(v)));

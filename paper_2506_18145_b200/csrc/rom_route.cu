@@ -15,9 +15,9 @@
 namespace rom {
 namespace {
 
-constexpr int TOK = 128;    // tokens per block of route_logits_topk
-constexpr int EG = 8;       // experts accumulated per thread
-constexpr int DC = 64;      // d_model elements staged per step
+constexpr int RT = kChunkTokens;   // tokens per block of route_logits_topk = one routing chunk (lanes of a warp)
+constexpr int EG = 4;              // experts accumulated per thread (one warp = 32 tokens x EG experts)
+constexpr int DC = 64;             // d_model elements staged per step
 
 template <typename T> struct XRow;
 template <> struct XRow<__nv_bfloat16> { static constexpr int kStrideBytes = DC * 2 + 16; };
@@ -39,8 +39,11 @@ __device__ __forceinline__ void load8(const float* p, double (&xd)[8]) {
   xd[4] = b.x; xd[5] = b.y; xd[6] = b.z; xd[7] = b.w;
 }
 
+// One block = 32 tokens (one routing chunk).  Warp g accumulates experts [4g, 4g+4) for the 32 tokens
+// (lane = token): per element of d_model one x value from the lane's staged row and four router
+// weights broadcast from shared memory, four independent fp64 FMA chains, strictly ascending d.
 template <typename T>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(512)
 route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const float* __restrict__ b_r,
                   int T_tokens, int Dm, int E, int K, int gate_mode,
                   int32_t* __restrict__ topk_idx, float* __restrict__ gates,
@@ -49,15 +52,15 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
   const int groups = (E + EG - 1) / EG;
   const int Epad = groups * EG;
   constexpr int XS = XRow<T>::kStrideBytes;
-  unsigned char* xs = smem;                                        // [TOK][XS]
-  double* wsd = reinterpret_cast<double*>(smem + TOK * XS);        // [Epad][DC]
-  double* lg = wsd + Epad * DC;                                    // [TOK][Epad]
-  int32_t* idx_s = reinterpret_cast<int32_t*>(lg + TOK * Epad);    // [TOK][K]
+  unsigned char* xs = smem;                                        // [RT][XS]
+  double* wsd = reinterpret_cast<double*>(smem + RT * XS);         // [DC][Epad]
+  double* lg = wsd + DC * Epad;                                    // [RT][Epad]
+  int32_t* idx_s = reinterpret_cast<int32_t*>(lg + RT * Epad);     // [RT][K]
 
   const int tid = threadIdx.x;
-  const int tok = tid % TOK;
-  const int g = tid / TOK;
-  const int t0 = blockIdx.x * TOK;
+  const int tok = tid & 31;
+  const int g = tid >> 5;
+  const int t0 = blockIdx.x * RT;
   const int nthr = blockDim.x;
 
   double acc[EG];
@@ -69,9 +72,9 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
 
   for (int d0 = 0; d0 < Dm; d0 += DC) {
     __syncthreads();
-    // stage x[t0 .. t0+TOK) x [d0, d0+DC) as raw storage type, 16 bytes per thread-step
+    // stage x[t0 .. t0+RT) x [d0, d0+DC) as raw storage type, 16 bytes per thread-step
     constexpr int VPR = DC * (int)sizeof(T) / 16;      // 16-byte vectors per row
-    for (int v = tid; v < TOK * VPR; v += nthr) {
+    for (int v = tid; v < RT * VPR; v += nthr) {
       const int r = v / VPR, cv = v % VPR;
       uint4 val = make_uint4(0, 0, 0, 0);
       if (t0 + r < T_tokens)
@@ -80,19 +83,23 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
     }
     for (int v = tid; v < Epad * DC; v += nthr) {
       const int e = v / DC, d = v % DC;
-      wsd[v] = (e < E) ? (double)to_f32(W_r[(size_t)e * Dm + d0 + d]) : 0.0;
+      wsd[d * Epad + e] = (e < E) ? (double)to_f32(W_r[(size_t)e * Dm + d0 + d]) : 0.0;
     }
     __syncthreads();
     const T* xrow = reinterpret_cast<const T*>(xs + tok * XS);
-#pragma unroll 1
+    const double* wg = wsd + g * EG;
+#pragma unroll 2
     for (int d8 = 0; d8 < DC; d8 += 8) {
       double xd[8];
       load8(xrow + d8, xd);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-#pragma unroll
-        for (int e = 0; e < EG; ++e)
-          acc[e] = fma(xd[j], wsd[(g * EG + e) * DC + d8 + j], acc[e]);
+        const double2 w01 = *reinterpret_cast<const double2*>(wg + (d8 + j) * Epad);
+        const double2 w23 = *reinterpret_cast<const double2*>(wg + (d8 + j) * Epad + 2);
+        acc[0] = fma(xd[j], w01.x, acc[0]);
+        acc[1] = fma(xd[j], w01.y, acc[1]);
+        acc[2] = fma(xd[j], w23.x, acc[2]);
+        acc[3] = fma(xd[j], w23.y, acc[3]);
       }
     }
   }
@@ -101,7 +108,7 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
   for (int e = 0; e < EG; ++e) lg[tok * Epad + g * EG + e] = acc[e];
   __syncthreads();
 
-  if (tid < TOK) {
+  if (tid < RT) {
     const int t = t0 + tid;
     const double* l = lg + tid * Epad;
     if (t < T_tokens) {
@@ -135,19 +142,11 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
     } else {
       for (int k = 0; k < K; ++k) idx_s[tid * K + k] = -1;
     }
-  }
-  __syncthreads();
-  // per-chunk (32 tokens) histogram by warp ballots
-  const int warp = tid >> 5, lane = tid & 31;
-  if (warp < TOK / kChunkTokens) {
-    const int chunk = blockIdx.x * (TOK / kChunkTokens) + warp;
-    const int ltok = warp * kChunkTokens + lane;
-    if ((size_t)chunk * kChunkTokens < (size_t)T_tokens) {
-      for (int e = 0; e < E; ++e) {
-        int c = 0;
-        for (int k = 0; k < K; ++k) c += __popc(__ballot_sync(0xffffffffu, idx_s[ltok * K + k] == e));
-        if (lane == 0) chunk_counts[(size_t)chunk * E + e] = c;
-      }
+    // histogram of this chunk by warp ballots (warp 0 holds all 32 tokens)
+    for (int e = 0; e < E; ++e) {
+      int c = 0;
+      for (int k = 0; k < K; ++k) c += __popc(__ballot_sync(0xffffffffu, idx_s[tid * K + k] == e));
+      if (tid == 0) chunk_counts[(size_t)blockIdx.x * E + e] = c;
     }
   }
 }
@@ -279,11 +278,11 @@ cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, co
   cudaError_t err = cudaMemsetAsync(assign_of_row, 0xff, sizeof(int32_t) * lay.rows_max, st);
   if (err != cudaSuccess) return err;
 
-  const int threads = TOK * groups;
-  const int blocks = (T + TOK - 1) / TOK;
+  const int threads = RT * groups;
+  const int blocks = (T + RT - 1) / RT;
   const bool bf = c.dtype == ROM_BF16;
-  const size_t xs_bytes = (size_t)TOK * (bf ? XRow<__nv_bfloat16>::kStrideBytes : XRow<float>::kStrideBytes);
-  const size_t smem = xs_bytes + sizeof(double) * ((size_t)Epad * DC + (size_t)TOK * Epad) + sizeof(int32_t) * TOK * c.K;
+  const size_t xs_bytes = (size_t)RT * (bf ? XRow<__nv_bfloat16>::kStrideBytes : XRow<float>::kStrideBytes);
+  const size_t smem = xs_bytes + sizeof(double) * ((size_t)Epad * DC + (size_t)RT * Epad) + sizeof(int32_t) * RT * c.K;
   if (bf) {
     err = cudaFuncSetAttribute(route_logits_topk<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
