@@ -40,6 +40,28 @@ __device__ __forceinline__ void store_vec(float* p, const float (&v)[4]) {
   *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
 }
 
+// One 16-byte vector kept as loaded; converted to fp32 only when used.
+template <typename T> struct RawVec;
+template <> struct RawVec<__nv_bfloat16> {
+  uint4 q;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ __forceinline__ void zero() { q = make_uint4(0, 0, 0, 0); }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+template <> struct RawVec<float> {
+  float4 q;
+  __device__ __forceinline__ void load(const float* p) { q = __ldg(reinterpret_cast<const float4*>(p)); }
+  __device__ __forceinline__ void zero() { q = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+  __device__ __forceinline__ void get(float (&v)[4]) const { v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
+};
+
 // Sum over the K slots of a token of one 16-byte vector of a [rows, ld] matrix (fp32 accumulation).
 template <typename T, int V, int KT>
 __device__ __forceinline__ void load_sum(const T* M, int ld, const int32_t* row_of_assign, int K, size_t t, int c0, float (&h)[V]) {
@@ -76,16 +98,41 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
   const int ld = 2 * De;
   const size_t tok0 = (size_t)b * L;
 
-  float hrow[TCH + 3][V];                 // rows tb-3 .. tb+TCH-1
+  // rows tb-3 .. tb+TCH-1 of H.  K = 1: kept as raw 16-byte words (row indices first, then all rows in
+  // flight at once) and converted on use; K > 1: summed over the slots as they arrive.
+  constexpr int NR = TCH + 3;
+  RawVec<T> raw[KT == 1 ? NR : 1];
+  float hsum[KT == 1 ? 1 : NR][V];
+  if constexpr (KT == 1) {
+    int32_t rix[NR];
 #pragma unroll
-  for (int r = 0; r < TCH + 3; ++r) {
-    const int t = tb - 3 + r;
-    if (t >= 0 && t < L) load_sum<T, V, KT>(XZp, ld, row_of_assign, K, tok0 + t, c0, hrow[r]);
-    else {
+    for (int r = 0; r < NR; ++r) {
+      const int t = tb - 3 + r;
+      rix[r] = (t >= 0 && t < L) ? __ldg(row_of_assign + tok0 + t) : -1;
+    }
 #pragma unroll
-      for (int i = 0; i < V; ++i) hrow[r][i] = 0.0f;
+    for (int r = 0; r < NR; ++r) {
+      if (rix[r] >= 0) raw[r].load(XZp + (size_t)rix[r] * ld + c0);
+      else raw[r].zero();
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < NR; ++r) {
+      const int t = tb - 3 + r;
+      if (t >= 0 && t < L) load_sum<T, V, KT>(XZp, ld, row_of_assign, K, tok0 + t, c0, hsum[r]);
+      else {
+#pragma unroll
+        for (int i = 0; i < V; ++i) hsum[r][i] = 0.0f;
+      }
     }
   }
+  auto hrow = [&](int r, float (&out)[V]) {
+    if constexpr (KT == 1) raw[r].get(out);
+    else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) out[i] = hsum[r][i];
+    }
+  };
   // taps right-aligned into 4 slots: slot 3 multiplies the current token
   float w[4][V];
 #pragma unroll
@@ -105,14 +152,15 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
   for (int r = 0; r < TCH; ++r) {
     const int t = tb + r;
     if (t >= L) break;
-    float u[V];
+    float u[V], h0[V], h1[V], h2[V], h3[V];
+    hrow(r, h0); hrow(r + 1, h1); hrow(r + 2, h2); hrow(r + 3, h3);
 #pragma unroll
     for (int i = 0; i < V; ++i) {
       float pre = bias[i];
-      pre = fmaf(w[0][i], hrow[r][i], pre);
-      pre = fmaf(w[1][i], hrow[r + 1][i], pre);
-      pre = fmaf(w[2][i], hrow[r + 2][i], pre);
-      pre = fmaf(w[3][i], hrow[r + 3][i], pre);
+      pre = fmaf(w[0][i], h0[i], pre);
+      pre = fmaf(w[1][i], h1[i], pre);
+      pre = fmaf(w[2][i], h2[i], pre);
+      pre = fmaf(w[3][i], h3[i], pre);
       u[i] = sizeof(T) == 2 ? silu_fast(pre) : silu_f(pre);
     }
     store_vec(U + (tok0 + t) * De + c0, u);

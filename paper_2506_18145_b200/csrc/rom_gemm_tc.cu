@@ -8,10 +8,12 @@
 // the per-expert Conv/Gate projection and Out projection of Section 4.2 (dropless, Section 5.1); with
 // one "expert" it also serves the shared x Proj / dt Proj.
 //
-// One persistent CTA per SM, 192 threads:
+// One persistent CTA per SM, 320 threads:
 //   warp 0      TMA producer: A tile 128x64 and B tile block_n x 64 per stage, 128-byte swizzle
 //   warp 1      allocates TMEM, issues tcgen05.mma (one thread), commits to mbarriers
-//   warps 2..5  epilogue: tcgen05.ld of the 128 x block_n fp32 accumulator, fused output op, stores
+//   warps 2..9  epilogue: tcgen05.ld of the 128 x block_n fp32 accumulator, fused output op, stores;
+//               two warps share each 32-lane quarter of tensor memory and take alternate 32-column
+//               chunks, and the load of the next chunk is in flight while one chunk is processed
 // The accumulator is double-buffered in TMEM (2 x 256 columns) so the epilogue of tile i overlaps
 // the MMAs of tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches an error code in
 // the status word, drains its own copies with a bounded wait, frees its TMEM and returns.
@@ -34,7 +36,8 @@ constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;      // 32 KB
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int ACC_STAGES = 2;
 constexpr int TMEM_COLS = 512;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait polls before a wait gives up (a few seconds)
 
@@ -83,7 +86,7 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -93,7 +96,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Waits for the outstanding tensor-memory load; the loaded registers pass through the statement so that
+// nothing that reads them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :: "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements),
@@ -109,32 +121,47 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   return d;
 }
 
-// Fused output op on one row segment of 8 consecutive columns (n0 % 8 == 0).
-__device__ __forceinline__ void epi_store8(const Epilogue& ep, size_t m, int n0, const float (&v)[8]) {
-  if (ep.mode == EPI_STORE || (ep.mode == EPI_XPROJ && n0 < ep.R)) {
-    const int ld = ep.mode == EPI_STORE ? ep.ldc : ep.R;
-    uint4 q;
-    uint32_t* w = reinterpret_cast<uint32_t*>(&q);
+// Fused output op on 32 consecutive accumulator columns [n0, n0+32) of row m (n0 % 32 == 0); columns at
+// or beyond N are skipped in groups of 8 (N % 8 == 0).
+template <int MODE>
+__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0, int N, const uint32_t (&r)[32]) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-      w[i] = *reinterpret_cast<uint32_t*>(&h);
+  for (int j = 0; j < 32; j += 8) {
+    const int n = n0 + j;
+    if (n >= N) break;
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j + i]);
+    if (MODE == EPI_STORE || (MODE == EPI_XPROJ && n < ep.R)) {
+      const int ld = MODE == EPI_STORE ? ep.ldc : ep.R;
+      uint4 q;
+      uint32_t* w = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + m * ld + n) = q;
+    } else if (MODE == EPI_XPROJ) {
+      float* dst = (n < ep.R + ep.N) ? ep.Bm + m * ep.N + (n - ep.R) : ep.Cm + m * ep.N + (n - ep.R - ep.N);
+      *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+    } else {
+      float4 b0 = make_float4(0.0f, 0.0f, 0.0f, 0.0f), b1 = b0;
+      if (ep.bias) {
+        b0 = __ldg(reinterpret_cast<const float4*>(ep.bias + n));
+        b1 = __ldg(reinterpret_cast<const float4*>(ep.bias + n) + 1);
+      }
+      float* dst = reinterpret_cast<float*>(ep.C) + m * ep.ldc + n;
+      *reinterpret_cast<float4*>(dst) = make_float4(softplus_fast(v[0] + b0.x), softplus_fast(v[1] + b0.y),
+                                                    softplus_fast(v[2] + b0.z), softplus_fast(v[3] + b0.w));
+      *reinterpret_cast<float4*>(dst + 4) = make_float4(softplus_fast(v[4] + b1.x), softplus_fast(v[5] + b1.y),
+                                                        softplus_fast(v[6] + b1.z), softplus_fast(v[7] + b1.w));
     }
-    *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + m * ld + n0) = q;
-  } else if (ep.mode == EPI_XPROJ) {
-    float* dst = (n0 < ep.R + ep.N) ? ep.Bm + m * ep.N + (n0 - ep.R) : ep.Cm + m * ep.N + (n0 - ep.R - ep.N);
-    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
-  } else {
-    float o[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) o[i] = softplus_fast(v[i] + (ep.bias ? __ldg(ep.bias + n0 + i) : 0.0f));
-    float* dst = reinterpret_cast<float*>(ep.C) + m * ep.ldc + n0;
-    *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[1], o[2], o[3]);
-    *reinterpret_cast<float4*>(dst + 4) = make_float4(o[4], o[5], o[6], o[7]);
   }
 }
 
+template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M_max, int N, int Kd, int block_n, uint32_t idesc,
@@ -164,7 +191,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), NUM_EPI_WARPS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -246,8 +273,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
+    const int half = (warp - 2) >> 2;             // which of the two warps of the quarter: takes chunks half, half+2, ...
+    const int n_chunks = block_n >> 5;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
@@ -256,21 +285,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tc_fence_after();
       const int row = m_tile * BLOCK_M + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * MAX_BLOCK_N;
-      for (int c0 = 0; c0 < block_n; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c0, r);
-        if (row < M_valid) {
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            const int n0 = n_tile * block_n + c0 + j;
-            if (n0 < N) {
-              float v[8];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j + i]);
-              epi_store8(ep, (size_t)row, n0, v);
-            }
-          }
-        }
+      const int n_base = n_tile * block_n;
+      uint32_t ra[32], rb[32];
+      int ch = half;
+      if (ch < n_chunks) tmem_ld32_issue(taddr + ch * 32, ra);
+      // two register buffers: while one chunk is processed the next chunk's tensor-memory load is in flight
+      while (ch < n_chunks) {
+        tmem_ld_wait(ra);
+        if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
+        if (row < M_valid) epi_store32<MODE>(ep, (size_t)row, n_base + ch * 32, N, ra);
+        ch += 2;
+        if (ch >= n_chunks) break;
+        tmem_ld_wait(rb);
+        if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
+        if (row < M_valid) epi_store32<MODE>(ep, (size_t)row, n_base + ch * 32, N, rb);
+        ch += 2;
       }
       tc_fence_before();
       __syncwarp();
@@ -340,12 +369,13 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ> : gemm_tc_kernel<EPI_SOFTPLUS>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int n_tiles = (N + block_n - 1) / block_n;
   const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
   const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
-  gemm_tc_kernel<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
+  kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
   count_launch();
   return cudaGetLastError();
 }

@@ -52,9 +52,9 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
   const int groups = (E + EG - 1) / EG;
   const int Epad = groups * EG;
   constexpr int XS = XRow<T>::kStrideBytes;
-  unsigned char* xs = smem;                                        // [RT][XS]
-  double* wsd = reinterpret_cast<double*>(smem + RT * XS);         // [DC][Epad]
-  double* lg = wsd + DC * Epad;                                    // [RT][Epad]
+  unsigned char* xs = smem;                                        // [2][RT][XS]   (double-buffered)
+  double* wsd = reinterpret_cast<double*>(smem + 2 * RT * XS);     // [2][DC][Epad]
+  double* lg = wsd + 2 * DC * Epad;                                // [RT][Epad]
   int32_t* idx_s = reinterpret_cast<int32_t*>(lg + RT * Epad);     // [RT][K]
 
   const int tid = threadIdx.x;
@@ -70,24 +70,48 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
     acc[e] = (b_r != nullptr && ee < E) ? (double)b_r[ee] : 0.0;
   }
 
-  for (int d0 = 0; d0 < Dm; d0 += DC) {
-    __syncthreads();
-    // stage x[t0 .. t0+RT) x [d0, d0+DC) as raw storage type, 16 bytes per thread-step
-    constexpr int VPR = DC * (int)sizeof(T) / 16;      // 16-byte vectors per row
+  // Chunk i+1 of x goes global -> shared with 16-byte asynchronous copies (rows past the end are
+  // zero-filled) and chunk i+1 of W_r is held in registers while chunk i is accumulated.
+  constexpr int VPR = DC * (int)sizeof(T) / 16;      // 16-byte vectors per row
+  constexpr int WPT = EG * DC / 32;                  // router weights per thread per chunk (Epad*DC / nthr)
+  auto copy_x = [&](int d0, int buf) {
     for (int v = tid; v < RT * VPR; v += nthr) {
       const int r = v / VPR, cv = v % VPR;
-      uint4 val = make_uint4(0, 0, 0, 0);
-      if (t0 + r < T_tokens)
-        val = *reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(x + (size_t)(t0 + r) * Dm + d0) + cv * 16);
-      *reinterpret_cast<uint4*>(xs + r * XS + cv * 16) = val;
+      const bool in = t0 + r < T_tokens;
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(x + (size_t)(in ? t0 + r : 0) * Dm + d0) + cv * 16;
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(xs + (buf * RT + r) * XS + cv * 16);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(in ? 16 : 0) : "memory");
     }
-    for (int v = tid; v < Epad * DC; v += nthr) {
-      const int e = v / DC, d = v % DC;
-      wsd[d * Epad + e] = (e < E) ? (double)to_f32(W_r[(size_t)e * Dm + d0 + d]) : 0.0;
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  float wpre[WPT];
+  auto fetch_w = [&](int d0) {
+#pragma unroll
+    for (int i = 0; i < WPT; ++i) {
+      const int v = tid + i * nthr, e = v / DC, d = v % DC;
+      wpre[i] = (e < E) ? to_f32(W_r[(size_t)e * Dm + d0 + d]) : 0.0f;
     }
-    __syncthreads();
-    const T* xrow = reinterpret_cast<const T*>(xs + tok * XS);
-    const double* wg = wsd + g * EG;
+  };
+  auto stash_w = [&](int buf) {
+#pragma unroll
+    for (int i = 0; i < WPT; ++i) {
+      const int v = tid + i * nthr, e = v / DC, d = v % DC;
+      wsd[(buf * DC + d) * Epad + e] = (double)wpre[i];
+    }
+  };
+
+  copy_x(0, 0);
+  fetch_w(0);
+  stash_w(0);
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  int buf = 0;
+  for (int d0 = 0; d0 < Dm; d0 += DC, buf ^= 1) {
+    const bool more = d0 + DC < Dm;
+    if (more) { copy_x(d0 + DC, buf ^ 1); fetch_w(d0 + DC); }
+    const T* xrow = reinterpret_cast<const T*>(xs + (buf * RT + tok) * XS);
+    const double* wg = wsd + buf * DC * Epad + g * EG;
 #pragma unroll 2
     for (int d8 = 0; d8 < DC; d8 += 8) {
       double xd[8];
@@ -102,6 +126,9 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
         acc[3] = fma(xd[j], w23.y, acc[3]);
       }
     }
+    if (more) stash_w(buf ^ 1);
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
   }
   __syncthreads();
 #pragma unroll
@@ -282,7 +309,7 @@ cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, co
   const int blocks = (T + RT - 1) / RT;
   const bool bf = c.dtype == ROM_BF16;
   const size_t xs_bytes = (size_t)RT * (bf ? XRow<__nv_bfloat16>::kStrideBytes : XRow<float>::kStrideBytes);
-  const size_t smem = xs_bytes + sizeof(double) * ((size_t)Epad * DC + (size_t)RT * Epad) + sizeof(int32_t) * RT * c.K;
+  const size_t smem = 2 * xs_bytes + sizeof(double) * (2 * (size_t)Epad * DC + (size_t)RT * Epad) + sizeof(int32_t) * RT * c.K;
   if (bf) {
     err = cudaFuncSetAttribute(route_logits_topk<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
