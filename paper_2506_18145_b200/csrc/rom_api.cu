@@ -42,6 +42,7 @@ WsLayout make_layout(const rom_config& c) {
   l.Delta = take(sizeof(float) * (size_t)l.T * c.d_inner);
   l.Ygp = take(l.esz * (size_t)l.rows_max * c.d_inner);
   l.Op = take(l.esz * (size_t)l.rows_max * c.d_model);
+  l.scan_ws = take(sizeof(float) * scan_ws_floats(c.B, c.d_inner, c.L));
   l.total = o;
   return l;
 }
@@ -148,7 +149,6 @@ int rom_route(const rom_config* cfg, const void* x, const void* W_r, const float
 
 int rom_scan(const rom_config* cfg, const void* u, const float* delta, const float* A, const float* Bm, const float* Cm,
              const float* D, const void* z, const float* h0, void* y, float* h_last, void* ws, size_t ws_bytes, void* stream) {
-  (void)ws; (void)ws_bytes;
   int rc = check_config(cfg, 2);
   if (rc != ROM_OK) return rc;
   if (!u || !delta || !A || !Bm || !Cm || !y) return ROM_ERR_INVALID_ARG;
@@ -158,7 +158,18 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
   if ((rc = check_device()) != ROM_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   LaunchCounter::count = 0;
-  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, st));
+  // with a workspace of rom_workspace_size bytes a long sequence is scanned in parallel chunks; without one, in one pass
+  float* chunk_ws = nullptr;
+  if (ws != nullptr) {
+    if (!aligned16(ws)) return ROM_ERR_INVALID_ARG;
+    rom_config full = *cfg;
+    if (full.E < 1) full.E = 1;
+    if (full.K < 1) full.K = 1;
+    const WsLayout lay = make_layout(full);
+    if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
+    chunk_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + lay.scan_ws);
+  }
+  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, chunk_ws, st));
   return ROM_OK;
 }
 
@@ -236,7 +247,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;
   ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
                        reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, c.K == 1 ? row_of_assign : nullptr,
-                       nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, st));
+                       nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), st));
   ROM_STAGE_DONE();
   // S10: grouped Out Proj
   Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0};

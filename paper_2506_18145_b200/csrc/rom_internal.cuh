@@ -21,11 +21,28 @@ constexpr int kStatWhere = 1;      // which wait gave up (debug aid)
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Chunks per sequence of the selective scan: 1 when batch x channels already gives the GPU about 2048 warps at
+// 8 states per thread, else enough chunks (at most 16, each at least 256 steps) to get there.  A function of
+// the problem sizes only, so that workspace sizing and the launch agree.
+inline int scan_chunks(int B, int De, int L) {
+  const long long warps1 = (long long)B * ((De + 127) / 128) * 8;
+  if (warps1 >= 2048) return 1;
+  long long n = (2048 + warps1 - 1) / warps1;
+  if (n > 16) n = 16;
+  while (n > 1 && (L + n - 1) / n < 256) --n;
+  return (int)n;
+}
+inline int scan_chunk_len(int L, int nch) { return (int)align_up((size_t)(L + nch - 1) / nch, 64); }
+inline size_t scan_ws_floats(int B, int De, int L) {
+  const int nch = scan_chunks(B, De, L);
+  return nch == 1 ? 0 : (size_t)B * nch * De * (2 * 16 + 1);
+}
+
 // Workspace carving, identical for every entry point (host arithmetic only).
 struct WsLayout {
   size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts;
   size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
-  size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op;
+  size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op, scan_ws;
   size_t total;
   int64_t T, A, rows_max, max_m_tiles, n_chunks;
   size_t esz;
@@ -74,9 +91,11 @@ cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row
 // Scan.  z is a [rows, ldz] matrix; the gate row of token t is z_row[t] (z_row == nullptr: row t).
 // y_rows == nullptr: y is [T, d_inner]; otherwise the output row of token t is written K times, to rows
 // y_rows[t*K + k].
+// chunk_ws == nullptr: one pass per sequence.  Otherwise a long sequence with too few channels to fill the GPU
+// is cut into scan_chunks() chunks scanned in parallel (two passes); chunk_ws holds scan_ws_floats() floats.
 cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
-                        void* y, float* h_last, const int32_t* y_rows, int K, cudaStream_t st);
+                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, cudaStream_t st);
 
 cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,
                            void* out, cudaStream_t st);

@@ -10,6 +10,13 @@
 // launcher picks the largest work per thread that still fills the GPU (small NS only for a single
 // long sequence).
 //
+// A single long sequence does not have enough (channel, state) lanes for the efficient shapes, so
+// the sequence is then cut into chunks that run in parallel, in two passes: pass 1 scans every chunk
+// from a zero state and keeps only its final state and sum of Delta; a small kernel chains the
+// chunk states (h_in[j+1] = exp(A sum_j Delta) h_in[j] + h_end[j], exact because the recurrence is
+// linear in h); pass 2 is the full scan of every chunk from its true initial state.  The
+// exponentials are evaluated twice; in exchange every SM runs the shape that keeps its pipes busy.
+//
 // A block of 256 threads owns CH = NC*256/S channels of one sequence and walks the sequence in tiles
 // of TS = 2048/CH steps, so every thread also owns one (row, 8 channels) piece of each tile: it
 // fetches that piece of tile i+1 (Delta, u, z) from global memory into registers -- raw,
@@ -105,12 +112,15 @@ struct ScanArgs {
   const void* u; const float* delta; const float* A; const float* Bm; const float* Cm; const float* D;
   const void* z; int ldz; const int32_t* z_row; const float* h0; void* y; float* h_last; const int32_t* y_rows;
   int K, L, De;
+  int Lc, nch;          // chunk length and chunks per sequence (nch == 1: Lc == L); blockIdx.z = chunk
+  float* sum_delta;     // STATE_ONLY: [B*nch, De] sum of Delta over the chunk
 };
 
 // PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance); otherwise one ex2.approx per
 // state update (bf16 configurations, 2e-2 tolerance).
 // ZOH: zero-order-hold B-bar (disc_mode 0); otherwise B-bar = Delta B.
-template <typename T, int NC, int NS, bool PRECISE, bool ZOH>
+// STATE_ONLY: pass 1 of the chunked scan: no outputs, only h_last and sum_delta of every chunk.
+template <typename T, int NC, int NS, bool PRECISE, bool ZOH, bool STATE_ONLY>
 __global__ void __launch_bounds__(BLOCK, NS >= 8 ? 2 : 1)
 scan_kernel(const ScanArgs p) {
   using G = Geo<NC, NS>;
@@ -122,13 +132,15 @@ scan_kernel(const ScanArgs p) {
   float* ps_all = ysum + 2 * TS * YP;                                                       // [8 warps][STRIP]
 
   const T* __restrict__ u = static_cast<const T*>(p.u);
-  const T* __restrict__ z = static_cast<const T*>(p.z);
+  const T* __restrict__ z = STATE_ONLY ? nullptr : static_cast<const T*>(p.z);
   T* __restrict__ y = static_cast<T*>(p.y);
-  const int L = p.L, De = p.De, K = p.K;
+  const int De = p.De, K = p.K;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.y;
+  const int chunk = blockIdx.z;
+  const int L = min(p.Lc, p.L - chunk * p.Lc);            // steps of this chunk
+  const int b = blockIdx.y * p.nch + chunk;               // index of the (sequence, chunk) state
   const int c_base = blockIdx.x * CH;
-  const size_t tok0 = (size_t)b * L;
+  const size_t tok0 = (size_t)blockIdx.y * p.L + (size_t)chunk * p.Lc;
 
   // ---- compute role: NC adjacent channels from block-local channel cl, states [g*NS, g*NS+NS)
   const int cl = (tid / S) * NC, g = tid % S;
@@ -149,6 +161,9 @@ scan_kernel(const ScanArgs p) {
     }
   }
   float* ps = ps_all + warp * G::STRIP;
+  float sdel[NC];
+#pragma unroll
+  for (int i = 0; i < NC; ++i) sdel[i] = 0.0f;
 
   // ---- loader / finisher role: row lr of every tile, channels [lc, lc + 8)
   const int lr = tid / G::CG, lc = (tid % G::CG) * 8;
@@ -252,6 +267,7 @@ scan_kernel(const ScanArgs p) {
       for (int i = 0; i < NC; ++i) {
         const float4 dv = dvp[tt * CH + cl_sw[i]];
         const float2 dl2 = make_float2(dv.x, dv.y), vv2 = make_float2(dv.z, dv.w);
+        if (STATE_ONLY) sdel[i] += dv.x;
         float2 acc0 = make_float2(0.0f, 0.0f), acc1 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int q = 0; q < NP; ++q) {
@@ -263,8 +279,10 @@ scan_kernel(const ScanArgs p) {
             const float w1 = ZOH ? -expm1f(dA1) * kin[i][q].y * Bv.y * vv2.x : Bv.y * vv2.x;
             h[i][q].x = fmaf(expf(dA0), h[i][q].x, w0);
             h[i][q].y = fmaf(expf(dA1), h[i][q].y, w1);
-            acc0.x = fmaf(Cv.x, h[i][q].x, acc0.x);
-            acc0.y = fmaf(Cv.y, h[i][q].y, acc0.y);
+            if (!STATE_ONLY) {
+              acc0.x = fmaf(Cv.x, h[i][q].x, acc0.x);
+              acc0.y = fmaf(Cv.y, h[i][q].y, acc0.y);
+            }
           } else {
             const float2 x = __fmul2_rn(dl2, a2[i][q]);
             const float2 a = make_float2(ex2_approx(x.x), ex2_approx(x.y));
@@ -276,14 +294,18 @@ scan_kernel(const ScanArgs p) {
             } else {
               h[i][q] = __ffma2_rn(a, h[i][q], __fmul2_rn(vv2, Bv));      // w = (Delta u) B
             }
-            float2& acc = (q & 1) ? acc1 : acc0;
-            acc = q < 2 ? __fmul2_rn(Cv, h[i][q]) : __ffma2_rn(Cv, h[i][q], acc);
+            if (!STATE_ONLY) {
+              float2& acc = (q & 1) ? acc1 : acc0;
+              acc = q < 2 ? __fmul2_rn(Cv, h[i][q]) : __ffma2_rn(Cv, h[i][q], acc);
+            }
           }
         }
         if (NP > 1 && !PRECISE) acc0 = __fadd2_rn(acc0, acc1);
         part[i] = acc0.x + acc0.y;
       }
-      if (S == 1) {
+      if (STATE_ONLY) {
+        // nothing to store: only the state and the sum of Delta leave this pass
+      } else if (S == 1) {
 #pragma unroll
         for (int i = 0; i < NC; ++i) ysp[tt * YP + i] = part[i];
       } else if (S <= 4) {
@@ -317,8 +339,10 @@ scan_kernel(const ScanArgs p) {
 
     if (more) stash(tiles[buf ^ 1]);
     __syncthreads();
-    flush(t0, ys);
-    if (more) { cur_u = pre_u; cur_z = pre_z; }
+    if (!STATE_ONLY) {
+      flush(t0, ys);
+      if (more) { cur_u = pre_u; cur_z = pre_z; }
+    }
   }
 
   if (p.h_last) {
@@ -332,18 +356,41 @@ scan_kernel(const ScanArgs p) {
         p.h_last[((size_t)b * De + c) * NST + n] = h[i][q].x;
         p.h_last[((size_t)b * De + c) * NST + n + 1] = h[i][q].y;
       }
+      if (STATE_ONLY && g == 0) p.sum_delta[(size_t)b * De + c] = sdel[i];
     }
   }
 }
 
-template <typename T, int NC, int NS, bool PRECISE, bool ZOH>
-cudaError_t launch_one(const ScanArgs& a, int B, cudaStream_t st) {
+// h_in of every chunk from the chunk-local end states: for each (sequence, channel, state), in chunk order,
+// h_in[j] = h;  h = exp(A * sum_delta[j]) * h + h_end[j].   One thread per (sequence, channel, state).
+__global__ void __launch_bounds__(256)
+chain_chunk_states(const float* __restrict__ A, const float* __restrict__ h0, const float* __restrict__ h_end,
+                   const float* __restrict__ sum_delta, float* __restrict__ h_in, float* __restrict__ h_last,
+                   int B, int De, int nch, int n_end) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)B * De * NST) return;
+  const int n = (int)(i % NST);
+  const int c = (int)((i / NST) % De);
+  const int b = (int)(i / ((long long)NST * De));
+  const float a = A[(size_t)c * NST + n];
+  float h = h0 ? h0[i] : 0.0f;
+  for (int j = 0; j < nch; ++j) {
+    const size_t sq = (size_t)b * nch + j;
+    h_in[(sq * De + c) * NST + n] = h;
+    if (j < n_end) h = fmaf(expf(a * sum_delta[sq * De + c]), h, h_end[(sq * De + c) * NST + n]);
+  }
+  if (h_last) h_last[i] = h;
+}
+
+template <typename T, int NC, int NS, bool PRECISE, bool ZOH, bool STATE_ONLY>
+cudaError_t launch_one(const ScanArgs& a, int B, int grid_z, cudaStream_t st) {
   using G = Geo<NC, NS>;
   const size_t smem = 2 * sizeof(Tile<NC, NS>) + (2 * (size_t)G::TS * G::YP + (BLOCK / 32) * G::STRIP) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, NC, NS, PRECISE, ZOH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, NC, NS, PRECISE, ZOH, STATE_ONLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid((a.De + G::CH - 1) / G::CH, B);
-  scan_kernel<T, NC, NS, PRECISE, ZOH><<<grid, BLOCK, smem, st>>>(a);
+  dim3 grid((a.De + G::CH - 1) / G::CH, B, grid_z);
+  scan_kernel<T, NC, NS, PRECISE, ZOH, STATE_ONLY><<<grid, BLOCK, smem, st>>>(a);
+  count_launch();
   return cudaGetLastError();
 }
 
@@ -363,19 +410,50 @@ int pick_thread_shape(int B, int De, int num_sms) {
 template <typename T, bool PRECISE, bool ZOH>
 cudaError_t launch_shape(int shape, const ScanArgs& a, int B, cudaStream_t st) {
   switch (shape) {
-    case 208: return launch_one<T, 2, 8, PRECISE, ZOH>(a, B, st);
-    case 108: return launch_one<T, 1, 8, PRECISE, ZOH>(a, B, st);
-    case 104: return launch_one<T, 1, 4, PRECISE, ZOH>(a, B, st);
-    case 102: return launch_one<T, 1, 2, PRECISE, ZOH>(a, B, st);
+    case 208: return launch_one<T, 2, 8, PRECISE, ZOH, false>(a, B, a.nch, st);
+    case 108: return launch_one<T, 1, 8, PRECISE, ZOH, false>(a, B, a.nch, st);
+    case 104: return launch_one<T, 1, 4, PRECISE, ZOH, false>(a, B, a.nch, st);
+    case 102: return launch_one<T, 1, 2, PRECISE, ZOH, false>(a, B, a.nch, st);
     default: return cudaErrorInvalidValue;
   }
+}
+
+template <typename T, bool PRECISE>
+cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const float* h0, float* h_last,
+                          float* chunk_ws, int num_sms, cudaStream_t st) {
+  const bool zoh = c.disc_mode == 0;
+  const int nch = chunk_ws ? scan_chunks(c.B, c.d_inner, c.L) : 1;
+  if (nch == 1) {
+    a.Lc = c.L; a.nch = 1;
+    const int shape = pick_thread_shape(c.B, c.d_inner, num_sms);
+    return zoh ? launch_shape<T, PRECISE, true>(shape, a, c.B, st) : launch_shape<T, PRECISE, false>(shape, a, c.B, st);
+  }
+  // chunked, two passes, 8 states per thread
+  const size_t n_state = (size_t)c.B * nch * c.d_inner * NST;
+  float* h_end = chunk_ws;
+  float* h_in = chunk_ws + n_state;
+  float* sum_delta = chunk_ws + 2 * n_state;
+  a.Lc = scan_chunk_len(c.L, nch); a.nch = nch;
+  const int n_end = h_last ? nch : nch - 1;       // the last chunk's end state is only needed for h_last
+  ScanArgs p1 = a;
+  p1.h0 = nullptr; p1.h_last = h_end; p1.sum_delta = sum_delta; p1.z = nullptr; p1.y = nullptr;
+  cudaError_t e = zoh ? launch_one<T, 1, 8, PRECISE, true, true>(p1, c.B, n_end, st)
+                      : launch_one<T, 1, 8, PRECISE, false, true>(p1, c.B, n_end, st);
+  if (e != cudaSuccess) return e;
+  const long long n_thr = (long long)c.B * c.d_inner * NST;
+  chain_chunk_states<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(A, h0, h_end, sum_delta, h_in, h_last, c.B, c.d_inner, nch, n_end);
+  count_launch();
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  a.h0 = h_in; a.h_last = nullptr;
+  return zoh ? launch_one<T, 1, 8, PRECISE, true, false>(a, c.B, nch, st) : launch_one<T, 1, 8, PRECISE, false, false>(a, c.B, nch, st);
 }
 
 }  // namespace
 
 cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
-                        void* y, float* h_last, const int32_t* y_rows, int K, cudaStream_t st) {
+                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, cudaStream_t st) {
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
@@ -384,15 +462,9 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, 
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner};
-  const int shape = pick_thread_shape(c.B, c.d_inner, num_sms);
-  cudaError_t e;
-  if (c.dtype == ROM_BF16)
-    e = c.disc_mode == 0 ? launch_shape<__nv_bfloat16, false, true>(shape, a, c.B, st) : launch_shape<__nv_bfloat16, false, false>(shape, a, c.B, st);
-  else
-    e = c.disc_mode == 0 ? launch_shape<float, true, true>(shape, a, c.B, st) : launch_shape<float, true, false>(shape, a, c.B, st);
-  count_launch();
-  return e;
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, nullptr};
+  return c.dtype == ROM_BF16 ? launch_scan_t<__nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
+                             : launch_scan_t<float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
 }
 
 }  // namespace rom

@@ -70,7 +70,7 @@ def test_route_bit_exact_full_size_configs(name):
 
 
 # ---------------------------------------------------------------------------------------------- scan
-def run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed):
+def run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed, use_ws=False):
     q = synth.make_scan_inputs(B, L, De, 16, dtype, seed, with_z=with_z, with_h0=with_h0)
     if not with_D:
         q["D"] = None
@@ -78,7 +78,8 @@ def run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed):
     d = {k: (None if v is None else v.cuda()) for k, v in q.items()}
     y = torch.empty_like(d["u"])
     h_last = torch.empty((B, De, 16), dtype=torch.float32, device="cuda")
-    rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], d["h0"], y, h_last)
+    ws = rb.alloc_workspace(cfg) if use_ws else None      # with a workspace long sequences run as parallel chunks
+    rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], d["h0"], y, h_last, ws)
     torch.cuda.synchronize()
     Y, hl = O.selective_scan(np64(q["u"]), np64(q["delta"]), np64(q["A"]), np64(q["Bm"]), np64(q["Cm"]), np64(q["D"]),
                              np64(q["h0"]), disc_mode)
@@ -99,6 +100,20 @@ def test_scan_parity(dtype, disc_mode, B, L, De, with_z, with_h0, with_D):
     y, Y, hl, HL = run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed=9100 + L)
     assert_close(y, Y, TOL[dtype], "scan y")
     assert_close(hl, HL, 1e-4 if dtype == "f32" else 2e-3, "scan h_last")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("disc_mode", [0, 1])
+@pytest.mark.parametrize("B,L,De,with_z,with_h0,with_D", [
+    (1, 2048, 256, True, False, True),     # 8 chunks of 256 steps
+    (2, 1500, 192, True, True, True),      # ragged last chunk, initial state carried through the chunk chain
+    (1, 4100, 64, False, True, False),     # chunk length rounded up: trailing chunks are empty
+    (3, 100, 128, True, True, True),       # too short to chunk: the workspace is simply unused
+])
+def test_scan_parity_chunked(dtype, disc_mode, B, L, De, with_z, with_h0, with_D):
+    y, Y, hl, HL = run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed=9500 + L, use_ws=True)
+    assert_close(y, Y, TOL[dtype], "chunked scan y")
+    assert_close(hl, HL, 1e-4 if dtype == "f32" else 2e-3, "chunked scan h_last")
 
 
 def test_scan_long_memory_small_delta():
