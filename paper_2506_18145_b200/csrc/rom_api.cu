@@ -169,7 +169,7 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
     if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
     chunk_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + lay.scan_ws);
   }
-  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, chunk_ws, st));
+  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, chunk_ws, false, st));
   return ROM_OK;
 }
 
@@ -228,7 +228,8 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   };
 
   // S3: grouped [Conv Proj | Gate Proj]
-  Epilogue e_in{EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, 0, 0};
+  // K = 1: the Gate Proj half is stored activated (SiLU); K > 1: raw, the activation follows the sum over slots in S4
+  Epilogue e_in{c.K == 1 ? EPI_INPROJ : EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, De, 0};
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
   ROM_STAGE_DONE();
   // S4: un-permute + sum over selected experts + conv + SiLU
@@ -247,7 +248,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;
   ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
                        reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, c.K == 1 ? row_of_assign : nullptr,
-                       nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), st));
+                       nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), true, st));
   ROM_STAGE_DONE();
   // S10: grouped Out Proj
   Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0};

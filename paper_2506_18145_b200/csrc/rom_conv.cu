@@ -166,13 +166,15 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
     store_vec(U + (tok0 + t) * De + c0, u);
   }
   if (Zs != nullptr) {
-    // gate pre-activation summed over the selected experts (indicator only), one row per token
+    // G = SiLU(sum over the selected experts of the Gate Proj rows) (indicator only), one row per token
 #pragma unroll
     for (int r = 0; r < TCH; ++r) {
       const int t = tb + r;
       if (t >= L) break;
       float zsum[V];
       load_sum<T, V, KT>(XZp + De, ld, row_of_assign, K, tok0 + t, c0, zsum);
+#pragma unroll
+      for (int i = 0; i < V; ++i) zsum[i] = sizeof(T) == 2 ? silu_fast(zsum[i]) : silu_f(zsum[i]);
       store_vec(Zs + (tok0 + t) * De + c0, zsum);
     }
   }

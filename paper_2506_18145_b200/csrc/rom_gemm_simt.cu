@@ -14,6 +14,9 @@ __device__ __forceinline__ void epi_store_scalar(const Epilogue& ep, int m, int 
     case EPI_STORE:
       reinterpret_cast<T*>(ep.C)[(size_t)m * ep.ldc + n] = from_f32<T>(v);
       break;
+    case EPI_INPROJ:
+      reinterpret_cast<T*>(ep.C)[(size_t)m * ep.ldc + n] = from_f32<T>(n >= ep.R ? silu_f(v) : v);
+      break;
     case EPI_XPROJ:
       if (n < ep.R) reinterpret_cast<T*>(ep.C)[(size_t)m * ep.R + n] = from_f32<T>(v);
       else if (n < ep.R + ep.N) ep.Bm[(size_t)m * ep.N + (n - ep.R)] = v;

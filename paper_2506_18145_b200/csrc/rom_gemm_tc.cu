@@ -132,8 +132,12 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
     float v[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[j + i]);
-    if (MODE == EPI_STORE || (MODE == EPI_XPROJ && n < ep.R)) {
-      const int ld = MODE == EPI_STORE ? ep.ldc : ep.R;
+    if (MODE == EPI_INPROJ && n >= ep.R) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = silu_fast(v[i]);
+    }
+    if (MODE == EPI_STORE || MODE == EPI_INPROJ || (MODE == EPI_XPROJ && n < ep.R)) {
+      const int ld = MODE == EPI_XPROJ ? ep.R : ep.ldc;
       uint4 q;
       uint32_t* w = reinterpret_cast<uint32_t*>(&q);
 #pragma unroll
@@ -369,7 +373,8 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ> : gemm_tc_kernel<EPI_SOFTPLUS>;
+  auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
+              : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : gemm_tc_kernel<EPI_SOFTPLUS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int n_tiles = (N + block_n - 1) / block_n;

@@ -22,15 +22,22 @@ constexpr int kStatWhere = 1;      // which wait gave up (debug aid)
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Chunks per sequence of the selective scan: 1 when batch x channels already gives the GPU about 2048 warps at
-// 8 states per thread, else enough chunks (at most 16, each at least 256 steps) to get there.  A function of
-// the problem sizes only, so that workspace sizing and the launch agree.
+// 8 states per thread; else the chunk count (at most 24, each at least 256 steps) whose blocks best fill whole
+// waves of two 256-thread blocks per SM (148 SMs assumed for sizing).  A function of the problem sizes only, so
+// that workspace sizing and the launch agree.
 inline int scan_chunks(int B, int De, int L) {
-  const long long warps1 = (long long)B * ((De + 127) / 128) * 8;
-  if (warps1 >= 2048) return 1;
-  long long n = (2048 + warps1 - 1) / warps1;
-  if (n > 16) n = 16;
-  while (n > 1 && (L + n - 1) / n < 256) --n;
-  return (int)n;
+  const long long blocks1 = (long long)B * ((De + 127) / 128);
+  if (blocks1 * 8 >= 2048) return 1;
+  const long long cap = 2 * 148;
+  int best = 1;
+  double best_fill = 0.0;
+  for (int n = 2; n <= 24 && (L + n - 1) / n >= 256; ++n) {
+    const long long blocks = blocks1 * n;
+    if (blocks * 8 < 2048 && n < 24 && (L + n) / (n + 1) >= 256) continue;      // still too few warps: keep growing
+    const double fill = (double)blocks / (double)(((blocks + cap - 1) / cap) * cap);
+    if (fill > best_fill + 1e-9) { best_fill = fill; best = n; }
+  }
+  return best;
 }
 inline int scan_chunk_len(int L, int nch) { return (int)align_up((size_t)(L + nch - 1) / nch, 64); }
 inline size_t scan_ws_floats(int B, int De, int L) {
@@ -56,7 +63,8 @@ inline void count_launch() { LaunchCounter::count++; }
 enum EpiMode : int {
   EPI_STORE = 0,      // C[m, n] = acc                          (dtype)
   EPI_XPROJ = 1,      // n < R: delta_r[m, n] (dtype); then Bm[m, n-R], Cm[m, n-R-N] (fp32)
-  EPI_SOFTPLUS = 2    // Delta[m, n] = softplus(acc + bias[n])  (fp32)
+  EPI_SOFTPLUS = 2,   // Delta[m, n] = softplus(acc + bias[n])  (fp32)
+  EPI_INPROJ = 3      // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype)
 };
 struct Epilogue {
   int mode;
@@ -85,17 +93,19 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
                            int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
                            const Epilogue& epi, int32_t* status, cudaStream_t st);
 
+// Zs (K > 1 only): [T, d_inner], SiLU of the Gate Proj rows summed over the K slots.
 cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
                         const float* b_conv, void* U, void* Zs, cudaStream_t st);
 
 // Scan.  z is a [rows, ldz] matrix; the gate row of token t is z_row[t] (z_row == nullptr: row t).
 // y_rows == nullptr: y is [T, d_inner]; otherwise the output row of token t is written K times, to rows
 // y_rows[t*K + k].
+// gate_activated: z already holds SiLU of the gate pre-activation (the producer applied it).
 // chunk_ws == nullptr: one pass per sequence.  Otherwise a long sequence with too few channels to fill the GPU
 // is cut into scan_chunks() chunks scanned in parallel (two passes); chunk_ws holds scan_ws_floats() floats.
 cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
-                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, cudaStream_t st);
+                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st);
 
 cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,
                            void* out, cudaStream_t st);

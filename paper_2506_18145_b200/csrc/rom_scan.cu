@@ -114,6 +114,7 @@ struct ScanArgs {
   int K, L, De;
   int Lc, nch;          // chunk length and chunks per sequence (nch == 1: Lc == L); blockIdx.z = chunk
   float* sum_delta;     // STATE_ONLY: [B*nch, De] sum of Delta over the chunk
+  int gate_activated;   // z already holds SiLU(gate pre-activation): multiply only
 };
 
 // PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance); otherwise one ex2.approx per
@@ -225,9 +226,14 @@ scan_kernel(const ScanArgs p) {
     if (z) {
       float zz[8];
       cur_z.get(zz);
+      if (p.gate_activated) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
-        o[i] *= PRECISE ? zz[i] / (1.0f + expf(-zz[i])) : __fdividef(zz[i], 1.0f + __expf(-zz[i]));
+        for (int i = 0; i < 8; ++i) o[i] *= zz[i];
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          o[i] *= PRECISE ? zz[i] / (1.0f + expf(-zz[i])) : __fdividef(zz[i], 1.0f + __expf(-zz[i]));
+      }
     }
     const size_t tok = tok0 + t;
     if (p.y_rows == nullptr) {
@@ -453,7 +459,7 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
 
 cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
-                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, cudaStream_t st) {
+                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st) {
   static int num_sms = 0;
   if (num_sms == 0) {
     int dev = 0;
@@ -462,7 +468,7 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, 
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, nullptr};
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, nullptr, gate_activated ? 1 : 0};
   return c.dtype == ROM_BF16 ? launch_scan_t<__nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
                              : launch_scan_t<float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
 }
