@@ -35,7 +35,12 @@ UNIT = "tokens/s"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel from one
 # ncu capture, keyed by (stage, workload); None = not captured.  The summaries the figures come from
 # are the text files under profiles/.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # scan stage = pass 1 (372.7 MB) + pass 2 (660.9 MB) of the chunked scan; profiles/scan_long_ctx.md
+    ("scan", "long_ctx"): 1033.6e6,
+    # profiles/in_proj_long_ctx.md
+    ("in_proj", "long_ctx"): 614.4e6,
+}
 
 
 def load_peaks():
@@ -60,7 +65,8 @@ def algorithmic_work(s: synth.RomShape):
         "conv": ("hbm", (s.K + 1) * T * De * esz),
         "x_proj": ("hbm", T * De * esz + T * (R * esz + 2 * N * 4)),
         "dt_proj": ("hbm", T * R * esz + T * De * esz),
-        "scan": ("hbm", T * (4 * De * esz + 8 * N)),
+        # one exponential per (token, channel, state) on the special-function unit: the binding limit of the scan
+        "scan": ("alu", float(T) * De * N),
         "out_proj": ("tensor", 2.0 * A * De * Dm),
         "combine": ("hbm", (s.K + 1) * T * Dm * esz),
     }
@@ -331,6 +337,11 @@ def main():
             if bound == "tensor":
                 ach = amount / (t_ms * 1e-3) / 1e12
                 peak, unit = peaks["bf16_tflops"], "TFLOP/s"
+            elif bound == "alu":
+                # special-function unit: 16 results per clock per SM, 148 SMs, at the maximum SM clock
+                sm_max = (clocks or {}).get("sm_max_mhz") or 1965.0
+                ach = amount / (t_ms * 1e-3) / 1e9
+                peak, unit = 148 * 16 * sm_max * 1e6 / 1e9, "Gexp/s"
             else:
                 ach = amount / (t_ms * 1e-3) / 1e9
                 peak, unit = peaks["hbm_gbs"], "GB/s"
@@ -340,13 +351,15 @@ def main():
         k = kernels[dom]
         roofline = {"kernel": dom, "bound": k["bound"], "achieved": k["achieved"], "peak": k["peak"], "unit": k["unit"],
                     "frac": k["frac"], "traffic": NCU_TRAFFIC_BYTES.get((dom, s.name)),
-                    "peak_source": f"of {peaks['source']} (burst bf16 / copy bandwidth)",
+                    "peak_source": (f"of {peaks['source']} (burst bf16 / copy bandwidth)" if k["bound"] != "alu" else
+                                    "derived: 16 exponentials per clock per SM x 148 SMs x max SM clock (unit rate checked by a microbenchmark)"),
                     "how": "CUDA events between stages on the launch stream, mean over profiled steps"}
-        # MUFU view of the scan: one ex2 per (token, channel, state) against 16 lanes/clk/SM * 148 SMs
-        if "scan" in stage_ms and clocks and clocks.get("sm_max_mhz"):
-            exps = s.T * s.d_inner * s.d_state
-            peak_exps = 148 * 16 * clocks["sm_max_mhz"] * 1e6
-            kernels["scan"]["alu_mufu_frac"] = round(exps / (stage_ms["scan"] * 1e-3) / peak_exps, 4)
+        # HBM view of the scan beside its special-function-unit roofline: u, Delta, z, y at storage width + B, C
+        if "scan" in stage_ms:
+            esz = 2 if s.dtype == "bf16" else 4
+            hb = s.T * (4 * s.d_inner * esz + 8 * s.d_state)
+            kernels["scan"]["hbm_achieved_gbs"] = round(hb / (stage_ms["scan"] * 1e-3) / 1e9, 2)
+            kernels["scan"]["hbm_frac"] = round(hb / (stage_ms["scan"] * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)
 
         tokens = s.T * world
         cpu = None
