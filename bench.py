@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-from paper_2506_18145_b200 import synth  # noqa: E402
+from paper_2506_18145_b200 import replicas, synth  # noqa: E402
 
 METRIC = "RoM layer fwd tokens/sec"
 UNIT = "tokens/s"
@@ -310,10 +310,7 @@ def main():
     barrier()
     ms_e2e = f0.elapsed_time(f1)
 
-    if dist is not None:
-        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = replicas.max_over_ranks([ms, ms_e2e], dist, dev)
 
     # ---- per-stage device times (CUDA events between the kernels, same stream, same inputs)
     stage_ms = {}
@@ -368,11 +365,11 @@ def main():
             dt, ntok, threads = oracle_sample(s, p, n_tok)
             cpu = {"value": ntok / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
                    "sample": f"first {ntok} tokens of sequence 0 of {s.name}, one run ({dt:.1f} s)"}
-        line = {"metric": METRIC, "value": tokens * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        line = {"metric": METRIC, "value": replicas.job_throughput(s.T, world, args.steps, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": workload_config(s), "clocks": clocks,
-                "e2e": {"value": tokens * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+                "e2e": {"value": replicas.job_throughput(s.T, world, args.steps, ms_e2e), "unit": UNIT,
                         "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
                         "d2h_bytes_per_step": out_host.numel() * out_host.element_size()},
                 "gpu_launches": launches_per_step * args.steps,
