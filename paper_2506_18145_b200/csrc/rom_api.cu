@@ -229,18 +229,18 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
 
   // S3: grouped [Conv Proj | Gate Proj]
   // K = 1: the Gate Proj half is stored activated (SiLU); K > 1: raw, the activation follows the sum over slots in S4
-  Epilogue e_in{c.K == 1 ? EPI_INPROJ : EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, De, 0};
+  Epilogue e_in{c.K == 1 ? EPI_INPROJ : EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, De, 0, nullptr, nullptr};
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
   ROM_STAGE_DONE();
   // S4: un-permute + sum over selected experts + conv + SiLU
   ROM_CUDA(launch_conv(c, W + lay.XZp, row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
   ROM_STAGE_DONE();
   // S5: x Proj -> delta_r | B | C
-  Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N};
+  Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N, nullptr, nullptr};
   ROM_CUDA(gemm(W + lay.U, De, w->W_x, De, 1, 0, T, R + 2 * N, De, nullptr, nullptr, e_x));
   ROM_STAGE_DONE();
   // S6: dt Proj + softplus
-  Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0};
+  Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0, nullptr, nullptr};
   ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
   ROM_STAGE_DONE();
   // S7 + S8 + S9: scan, gate, re-permute
@@ -250,13 +250,22 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
                        reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, c.K == 1 ? row_of_assign : nullptr,
                        nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), true, st));
   ROM_STAGE_DONE();
-  // S10: grouped Out Proj
-  Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0};
-  ROM_CUDA(gemm(W + lay.Ygp, De, w->W_out, De, c.E, (int64_t)Dm * De, (int)lay.rows_max, Dm, De, tile_expert, num_m_tiles, e_out));
-  ROM_STAGE_DONE();
-  // S11: gate-weighted combine
-  ROM_CUDA(launch_combine(c, W + lay.Op, row_of_assign, gates, out, st));
-  ROM_STAGE_DONE();
+  // S10 + S11.  Tensor path with one expert per token: the epilogue of the grouped Out Proj scales each row by
+  // its gate and writes it at its token's position (no intermediate rows, no combine pass).  Otherwise: grouped
+  // Out Proj into expert-order rows, then the gate-weighted sum over the K slots.
+  const bool fused_out = tc && c.K == 1;
+  if (fused_out) {
+    Epilogue e_out{EPI_OUTPROJ, out, Dm, nullptr, nullptr, nullptr, 0, 0, reinterpret_cast<const int32_t*>(W + lay.assign_of_row), gates};
+    ROM_CUDA(gemm(W + lay.Ygp, De, w->W_out, De, c.E, (int64_t)Dm * De, (int)lay.rows_max, Dm, De, tile_expert, num_m_tiles, e_out));
+    ROM_STAGE_DONE();
+    ROM_STAGE_DONE();
+  } else {
+    Epilogue e_out{EPI_STORE, W + lay.Op, Dm, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
+    ROM_CUDA(gemm(W + lay.Ygp, De, w->W_out, De, c.E, (int64_t)Dm * De, (int)lay.rows_max, Dm, De, tile_expert, num_m_tiles, e_out));
+    ROM_STAGE_DONE();
+    ROM_CUDA(launch_combine(c, W + lay.Op, row_of_assign, gates, out, st));
+    ROM_STAGE_DONE();
+  }
 #undef ROM_STAGE_DONE
   return ROM_OK;
 }

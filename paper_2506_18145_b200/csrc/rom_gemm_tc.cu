@@ -124,7 +124,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
 // Fused output op on 32 consecutive accumulator columns [n0, n0+32) of row m (n0 % 32 == 0); columns at
 // or beyond N are skipped in groups of 8 (N % 8 == 0).
 template <int MODE>
-__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0, int N, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0, int N, const uint32_t (&r)[32], float scale) {
 #pragma unroll
   for (int j = 0; j < 32; j += 8) {
     const int n = n0 + j;
@@ -136,7 +136,11 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
 #pragma unroll
       for (int i = 0; i < 8; ++i) v[i] = silu_fast(v[i]);
     }
-    if (MODE == EPI_STORE || MODE == EPI_INPROJ || (MODE == EPI_XPROJ && n < ep.R)) {
+    if (MODE == EPI_OUTPROJ) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] *= scale;
+    }
+    if (MODE == EPI_STORE || MODE == EPI_INPROJ || MODE == EPI_OUTPROJ || (MODE == EPI_XPROJ && n < ep.R)) {
       const int ld = MODE == EPI_XPROJ ? ep.R : ep.ldc;
       uint4 q;
       uint32_t* w = reinterpret_cast<uint32_t*>(&q);
@@ -288,6 +292,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int row = m_tile * BLOCK_M + quarter * 32 + lane;
+      bool row_ok = row < M_valid;
+      size_t out_row = (size_t)row;
+      float scale = 1.0f;
+      if (MODE == EPI_OUTPROJ && row_ok) {
+        const int tok = __ldg(ep.row_token + row);
+        row_ok = tok >= 0;
+        if (row_ok) { out_row = (size_t)tok; scale = __ldg(ep.row_scale + tok); }
+      }
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * MAX_BLOCK_N;
       const int n_base = n_tile * block_n;
       uint32_t ra[32], rb[32];
@@ -297,12 +309,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       while (ch < n_chunks) {
         tmem_ld_wait(ra);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
-        if (row < M_valid) epi_store32<MODE>(ep, (size_t)row, n_base + ch * 32, N, ra);
+        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale);
         ch += 2;
         if (ch >= n_chunks) break;
         tmem_ld_wait(rb);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
-        if (row < M_valid) epi_store32<MODE>(ep, (size_t)row, n_base + ch * 32, N, rb);
+        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale);
         ch += 2;
       }
       tc_fence_before();
@@ -374,7 +386,8 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
     if (e != cudaSuccess) return e;
   }
   auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
-              : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : gemm_tc_kernel<EPI_SOFTPLUS>;
+              : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : epi.mode == EPI_OUTPROJ ? gemm_tc_kernel<EPI_OUTPROJ>
+              : gemm_tc_kernel<EPI_SOFTPLUS>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int n_tiles = (N + block_n - 1) / block_n;

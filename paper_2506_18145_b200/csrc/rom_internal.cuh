@@ -64,7 +64,9 @@ enum EpiMode : int {
   EPI_STORE = 0,      // C[m, n] = acc                          (dtype)
   EPI_XPROJ = 1,      // n < R: delta_r[m, n] (dtype); then Bm[m, n-R], Cm[m, n-R-N] (fp32)
   EPI_SOFTPLUS = 2,   // Delta[m, n] = softplus(acc + bias[n])  (fp32)
-  EPI_INPROJ = 3      // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype)
+  EPI_INPROJ = 3,     // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype)
+  EPI_OUTPROJ = 4     // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
+                      // row_token[m] < 0 (segment padding) are skipped   (dtype; tensor path only)
 };
 struct Epilogue {
   int mode;
@@ -74,6 +76,8 @@ struct Epilogue {
   float* Cm;
   const float* bias;  // EPI_SOFTPLUS (may be null)
   int R, N;
+  const int32_t* row_token;   // EPI_OUTPROJ: token of each (padded) row, -1 in padding
+  const float* row_scale;     // EPI_OUTPROJ: gate of each token
 };
 
 // ---------------------------------------------------------------- launchers (each returns a cudaError_t)
@@ -118,13 +122,16 @@ template <> __device__ __forceinline__ float from_f32<float>(float v) { return v
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.0f + __expf(-v)); }
-// Fast forms for the bf16 path (results are rounded to bf16 or feed a 2e-2 tolerance): approximate
-// reciprocal / exp2 / log2 of the special-function unit, relative error ~1e-6.
-__device__ __forceinline__ float silu_fast(float v) { return __fdividef(v, 1.0f + __expf(-v)); }
+// Fast forms for the bf16 path (results are rounded to bf16 or feed a 2e-2 tolerance): the special-function
+// unit's approximate exp2 / log2 / reciprocal with flush-to-zero, relative error ~1e-6, no range fix-ups.
+__device__ __forceinline__ float ex2_ftz(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float lg2_ftz(float x) { float y; asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float rcp_ftz(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float silu_fast(float v) { return v * rcp_ftz(1.0f + ex2_ftz(-1.4426950408889634f * v)); }
 __device__ __forceinline__ float softplus_fast(float v) {
   // max(v,0) + log(1 + e), e = exp(-|v|) in (0, 1].  For tiny e, 1 + e loses e's low bits: use log1p(e) ~ e.
-  const float e = __expf(-fabsf(v));
-  const float l = e < 2.44140625e-4f ? e : __logf(1.0f + e);
+  const float e = ex2_ftz(-1.4426950408889634f * fabsf(v));
+  const float l = e < 2.44140625e-4f ? e : 0.6931471805599453f * lg2_ftz(1.0f + e);
   return fmaxf(v, 0.0f) + l;
 }
 __device__ __forceinline__ float softplus_f(float v) {

@@ -232,7 +232,7 @@ scan_kernel(const ScanArgs p) {
       } else {
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          o[i] *= PRECISE ? zz[i] / (1.0f + expf(-zz[i])) : __fdividef(zz[i], 1.0f + __expf(-zz[i]));
+          o[i] *= PRECISE ? zz[i] / (1.0f + expf(-zz[i])) : silu_fast(zz[i]);
       }
     }
     const size_t tok = tok0 + t;
