@@ -121,10 +121,21 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   return d;
 }
 
+// Bias of the 32 columns [n0, n0+32) (EPI_SOFTPLUS only), requested before the accumulator chunk is waited for.
+template <int MODE>
+__device__ __forceinline__ void load_bias(const Epilogue& ep, int n0, int N, float4 (&bq)[8]) {
+  if constexpr (MODE == EPI_SOFTPLUS) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      bq[i] = (ep.bias && n0 + 4 * i < N) ? __ldg(reinterpret_cast<const float4*>(ep.bias + n0) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+  }
+}
+
 // Fused output op on 32 consecutive accumulator columns [n0, n0+32) of row m (n0 % 32 == 0); columns at
 // or beyond N are skipped in groups of 8 (N % 8 == 0).
 template <int MODE>
-__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0, int N, const uint32_t (&r)[32], float scale) {
+__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0, int N, const uint32_t (&r)[32], float scale,
+                                            const float4 (&bq)[8]) {
 #pragma unroll
   for (int j = 0; j < 32; j += 8) {
     const int n = n0 + j;
@@ -155,11 +166,7 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
       *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
       *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
     } else {
-      float4 b0 = make_float4(0.0f, 0.0f, 0.0f, 0.0f), b1 = b0;
-      if (ep.bias) {
-        b0 = __ldg(reinterpret_cast<const float4*>(ep.bias + n));
-        b1 = __ldg(reinterpret_cast<const float4*>(ep.bias + n) + 1);
-      }
+      const float4 b0 = bq[j / 4], b1 = bq[j / 4 + 1];
       float* dst = reinterpret_cast<float*>(ep.C) + m * ep.ldc + n;
       *reinterpret_cast<float4*>(dst) = make_float4(softplus_fast(v[0] + b0.x), softplus_fast(v[1] + b0.y),
                                                     softplus_fast(v[2] + b0.z), softplus_fast(v[3] + b0.w));
@@ -303,18 +310,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * MAX_BLOCK_N;
       const int n_base = n_tile * block_n;
       uint32_t ra[32], rb[32];
+      float4 bq[8];
       int ch = half;
       if (ch < n_chunks) tmem_ld32_issue(taddr + ch * 32, ra);
       // two register buffers: while one chunk is processed the next chunk's tensor-memory load is in flight
       while (ch < n_chunks) {
+        load_bias<MODE>(ep, n_base + ch * 32, N, bq);     // in flight together with the tensor-memory load
         tmem_ld_wait(ra);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
-        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale);
+        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale, bq);
         ch += 2;
         if (ch >= n_chunks) break;
+        load_bias<MODE>(ep, n_base + ch * 32, N, bq);
         tmem_ld_wait(rb);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
-        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale);
+        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale, bq);
         ch += 2;
       }
       tc_fence_before();
