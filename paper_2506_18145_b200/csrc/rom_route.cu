@@ -53,7 +53,7 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
   const int Epad = groups * EG;
   constexpr int XS = XRow<T>::kStrideBytes;
   unsigned char* xs = smem;                                        // [2][RT][XS]   (double-buffered)
-  double* wsd = reinterpret_cast<double*>(smem + 2 * RT * XS);     // [2][DC][Epad]
+  double* wsd = reinterpret_cast<double*>(smem + 2 * RT * XS);     // [2][groups][DC][EG]: a warp's four experts of one d are adjacent
   double* lg = wsd + 2 * DC * Epad;                                // [RT][Epad]
   int32_t* idx_s = reinterpret_cast<int32_t*>(lg + RT * Epad);     // [RT][K]
 
@@ -96,7 +96,7 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
 #pragma unroll
     for (int i = 0; i < WPT; ++i) {
       const int v = tid + i * nthr, e = v / DC, d = v % DC;
-      wsd[(buf * DC + d) * Epad + e] = (double)wpre[i];
+      wsd[((buf * groups + e / EG) * DC + d) * EG + (e % EG)] = (double)wpre[i];
     }
   };
 
@@ -111,15 +111,15 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
     const bool more = d0 + DC < Dm;
     if (more) { copy_x(d0 + DC, buf ^ 1); fetch_w(d0 + DC); }
     const T* xrow = reinterpret_cast<const T*>(xs + (buf * RT + tok) * XS);
-    const double* wg = wsd + buf * DC * Epad + g * EG;
+    const double* wg = wsd + (buf * groups + g) * DC * EG;
 #pragma unroll 2
     for (int d8 = 0; d8 < DC; d8 += 8) {
       double xd[8];
       load8(xrow + d8, xd);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        const double2 w01 = *reinterpret_cast<const double2*>(wg + (d8 + j) * Epad);
-        const double2 w23 = *reinterpret_cast<const double2*>(wg + (d8 + j) * Epad + 2);
+        const double2 w01 = *reinterpret_cast<const double2*>(wg + (d8 + j) * EG);
+        const double2 w23 = *reinterpret_cast<const double2*>(wg + (d8 + j) * EG + 2);
         acc[0] = fma(xd[j], w01.x, acc[0]);
         acc[1] = fma(xd[j], w01.y, acc[1]);
         acc[2] = fma(xd[j], w23.x, acc[2]);

@@ -263,6 +263,7 @@ scan_kernel(const ScanArgs p) {
     float* __restrict__ ysp = ys + cl;
     float* __restrict__ psp = ps;
     constexpr int UF = S > 4 ? S : (NC * NS >= 16 ? 2 : 4);
+    float held = 0.0f;      // the even step's partial sum, kept for the paired exchange (S == 2)
 #pragma unroll UF
     for (int tt = 0; tt < TS; ++tt) {
       float4 bc[NP];
@@ -314,6 +315,15 @@ scan_kernel(const ScanArgs p) {
       } else if (S == 1) {
 #pragma unroll
         for (int i = 0; i < NC; ++i) ysp[tt * YP + i] = part[i];
+      } else if (S == 2 && NC == 1) {
+        // steps are finished in pairs with one exchange: lane 0 completes the even step (it needs the partner's
+        // even partial), lane 1 the odd step (it needs the partner's odd partial)
+        if ((tt & 1) == 0) {
+          held = part[0];
+        } else {
+          const float recv = __shfl_xor_sync(0xffffffffu, g ? held : part[0], 1);
+          ysp[(tt - 1 + g) * YP] = (g ? part[0] : held) + recv;
+        }
       } else if (S <= 4) {
         // all S lanes of the channel get the sum; lane g stores the steps with tt % S == g
 #pragma unroll
