@@ -22,9 +22,9 @@ constexpr int kStatWhere = 1;      // which wait gave up (debug aid)
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Chunks per sequence of the selective scan: 1 when batch x channels already gives the GPU about 2048 warps at
-// 8 states per thread; else the chunk count (at most 24, each at least 256 steps) whose blocks best fill whole
-// waves of two 256-thread blocks per SM (148 SMs assumed for sizing).  A function of the problem sizes only, so
-// that workspace sizing and the launch agree.
+// 8 states per thread; else the chunk count n (at most 24, each chunk at least 256 steps) for which the n - 1
+// chunks of each of the two launches best fill whole waves of two 256-thread blocks per SM (148 SMs assumed
+// for sizing).  A function of the problem sizes only, so that workspace sizing and the launch agree.
 inline int scan_chunks(int B, int De, int L) {
   const long long blocks1 = (long long)B * ((De + 127) / 128);
   if (blocks1 * 8 >= 2048) return 1;
@@ -32,7 +32,7 @@ inline int scan_chunks(int B, int De, int L) {
   int best = 1;
   double best_fill = 0.0;
   for (int n = 2; n <= 24 && (L + n - 1) / n >= 256; ++n) {
-    const long long blocks = blocks1 * n;
+    const long long blocks = blocks1 * (n - 1);
     if (blocks * 8 < 2048 && n < 24 && (L + n) / (n + 1) >= 256) continue;      // still too few warps: keep growing
     const double fill = (double)blocks / (double)(((blocks + cap - 1) / cap) * cap);
     if (fill > best_fill + 1e-9) { best_fill = fill; best = n; }

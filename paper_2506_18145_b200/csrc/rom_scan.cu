@@ -27,6 +27,8 @@
 // per-channel operands are stored duplicated, (Delta, Delta, v, v), so one 16-byte load yields both
 // packed operands; 8-channel groups are XOR-swizzled so that loader stores and compute loads are
 // both bank-conflict free.
+#include <type_traits>
+
 #include "rom_internal.cuh"
 
 namespace rom {
@@ -113,15 +115,18 @@ struct ScanArgs {
   const void* z; int ldz; const int32_t* z_row; const float* h0; void* y; float* h_last; const int32_t* y_rows;
   int K, L, De;
   int Lc, nch;          // chunk length and chunks per sequence (nch == 1: Lc == L); blockIdx.z = chunk
-  float* sum_delta;     // STATE_ONLY: [B*nch, De] sum of Delta over the chunk
+  float* sum_delta;     // state-only blocks: [B*nch, De] sum of Delta over the chunk
   int gate_activated;   // z already holds SiLU(gate pre-activation): multiply only
+  int chunk_off;        // chunk of blockIdx.z == 0
 };
 
 // PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance); otherwise one ex2.approx per
 // state update (bf16 configurations, 2e-2 tolerance).
 // ZOH: zero-order-hold B-bar (disc_mode 0); otherwise B-bar = Delta B.
-// STATE_ONLY: pass 1 of the chunked scan: no outputs, only h_last and sum_delta of every chunk.
-template <typename T, int NC, int NS, bool PRECISE, bool ZOH, bool STATE_ONLY>
+// MODE 0: full scan.  MODE 1: state only (no outputs, only h_last and sum_delta of every chunk).  MODE 2: first
+// launch of the chunked scan: chunk 0 runs the full scan from the caller's initial state (h0 indexed by
+// sequence), the other chunks run state-only from a zero state.
+template <typename T, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
 __global__ void __launch_bounds__(BLOCK, NS >= 8 ? 2 : 1)
 scan_kernel(const ScanArgs p) {
   using G = Geo<NC, NS>;
@@ -133,11 +138,13 @@ scan_kernel(const ScanArgs p) {
   float* ps_all = ysum + 2 * TS * YP;                                                       // [8 warps][STRIP]
 
   const T* __restrict__ u = static_cast<const T*>(p.u);
-  const T* __restrict__ z = STATE_ONLY ? nullptr : static_cast<const T*>(p.z);
+
   T* __restrict__ y = static_cast<T*>(p.y);
   const int De = p.De, K = p.K;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int chunk = blockIdx.z;
+  const int chunk = blockIdx.z + p.chunk_off;
+  const bool so = MODE == 1 || (MODE == 2 && chunk != 0);  // this block only produces its end state
+  const T* __restrict__ z = so ? nullptr : static_cast<const T*>(p.z);
   const int L = min(p.Lc, p.L - chunk * p.Lc);            // steps of this chunk
   const int b = blockIdx.y * p.nch + chunk;               // index of the (sequence, chunk) state
   const int c_base = blockIdx.x * CH;
@@ -157,8 +164,9 @@ scan_kernel(const ScanArgs p) {
       const float a0 = p.A[(size_t)c * NST + n], a1 = p.A[(size_t)c * NST + n + 1];
       a2[i][q] = PRECISE ? make_float2(a0, a1) : make_float2(a0 * kLog2e, a1 * kLog2e);
       kin[i][q] = make_float2(-1.0f / a0, -1.0f / a1);
-      h[i][q] = p.h0 ? make_float2(p.h0[((size_t)b * De + c) * NST + n], p.h0[((size_t)b * De + c) * NST + n + 1])
-                     : make_float2(0.0f, 0.0f);
+      const size_t hb = MODE == 2 ? (size_t)blockIdx.y : (size_t)b;
+      h[i][q] = (p.h0 && !(MODE == 2 && so)) ? make_float2(p.h0[(hb * De + c) * NST + n], p.h0[(hb * De + c) * NST + n + 1])
+                                             : make_float2(0.0f, 0.0f);
     }
   }
   float* ps = ps_all + warp * G::STRIP;
@@ -264,6 +272,8 @@ scan_kernel(const ScanArgs p) {
     float* __restrict__ psp = ps;
     constexpr int UF = S > 4 ? S : (NC * NS >= 16 ? 2 : 4);
     float held = 0.0f;      // the even step's partial sum, kept for the paired exchange (S == 2)
+    auto tile_steps = [&](auto so_tag) {
+    constexpr bool STATE_ONLY = decltype(so_tag)::value;
 #pragma unroll UF
     for (int tt = 0; tt < TS; ++tt) {
       float4 bc[NP];
@@ -353,9 +363,15 @@ scan_kernel(const ScanArgs p) {
       }
     }
 
+    };
+    if (MODE == 0) tile_steps(std::false_type{});
+    else if (MODE == 1) tile_steps(std::true_type{});
+    else if (so) tile_steps(std::true_type{});
+    else tile_steps(std::false_type{});
+
     if (more) stash(tiles[buf ^ 1]);
     __syncthreads();
-    if (!STATE_ONLY) {
+    if (!so) {
       flush(t0, ys);
       if (more) { cur_u = pre_u; cur_z = pre_z; }
     }
@@ -372,25 +388,25 @@ scan_kernel(const ScanArgs p) {
         p.h_last[((size_t)b * De + c) * NST + n] = h[i][q].x;
         p.h_last[((size_t)b * De + c) * NST + n + 1] = h[i][q].y;
       }
-      if (STATE_ONLY && g == 0) p.sum_delta[(size_t)b * De + c] = sdel[i];
+      if (so && g == 0) p.sum_delta[(size_t)b * De + c] = sdel[i];
     }
   }
 }
 
-// h_in of every chunk from the chunk-local end states: for each (sequence, channel, state), in chunk order,
-// h_in[j] = h;  h = exp(A * sum_delta[j]) * h + h_end[j].   One thread per (sequence, channel, state).
+// Initial state of every chunk after the first.  h_end[0] is the true state after chunk 0 (it ran from the
+// caller's h0); for j >= 1, h_end[j] is chunk j's end state from a zero start.  In chunk order, per
+// (sequence, channel, state):  h = h_end[0];  h_in[j] = h;  h = exp(A * sum_delta[j]) * h + h_end[j].
 __global__ void __launch_bounds__(256)
-chain_chunk_states(const float* __restrict__ A, const float* __restrict__ h0, const float* __restrict__ h_end,
-                   const float* __restrict__ sum_delta, float* __restrict__ h_in, float* __restrict__ h_last,
-                   int B, int De, int nch, int n_end) {
+chain_chunk_states(const float* __restrict__ A, const float* __restrict__ h_end, const float* __restrict__ sum_delta,
+                   float* __restrict__ h_in, float* __restrict__ h_last, int B, int De, int nch, int n_end) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= (long long)B * De * NST) return;
   const int n = (int)(i % NST);
   const int c = (int)((i / NST) % De);
   const int b = (int)(i / ((long long)NST * De));
   const float a = A[(size_t)c * NST + n];
-  float h = h0 ? h0[i] : 0.0f;
-  for (int j = 0; j < nch; ++j) {
+  float h = h_end[(((size_t)b * nch) * De + c) * NST + n];
+  for (int j = 1; j < nch; ++j) {
     const size_t sq = (size_t)b * nch + j;
     h_in[(sq * De + c) * NST + n] = h;
     if (j < n_end) h = fmaf(expf(a * sum_delta[sq * De + c]), h, h_end[(sq * De + c) * NST + n]);
@@ -398,14 +414,14 @@ chain_chunk_states(const float* __restrict__ A, const float* __restrict__ h0, co
   if (h_last) h_last[i] = h;
 }
 
-template <typename T, int NC, int NS, bool PRECISE, bool ZOH, bool STATE_ONLY>
+template <typename T, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
 cudaError_t launch_one(const ScanArgs& a, int B, int grid_z, cudaStream_t st) {
   using G = Geo<NC, NS>;
   const size_t smem = 2 * sizeof(Tile<NC, NS>) + (2 * (size_t)G::TS * G::YP + (BLOCK / 32) * G::STRIP) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, NC, NS, PRECISE, ZOH, STATE_ONLY>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, NC, NS, PRECISE, ZOH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((a.De + G::CH - 1) / G::CH, B, grid_z);
-  scan_kernel<T, NC, NS, PRECISE, ZOH, STATE_ONLY><<<grid, BLOCK, smem, st>>>(a);
+  scan_kernel<T, NC, NS, PRECISE, ZOH, MODE><<<grid, BLOCK, smem, st>>>(a);
   count_launch();
   return cudaGetLastError();
 }
@@ -426,10 +442,10 @@ int pick_thread_shape(int B, int De, int num_sms) {
 template <typename T, bool PRECISE, bool ZOH>
 cudaError_t launch_shape(int shape, const ScanArgs& a, int B, cudaStream_t st) {
   switch (shape) {
-    case 208: return launch_one<T, 2, 8, PRECISE, ZOH, false>(a, B, a.nch, st);
-    case 108: return launch_one<T, 1, 8, PRECISE, ZOH, false>(a, B, a.nch, st);
-    case 104: return launch_one<T, 1, 4, PRECISE, ZOH, false>(a, B, a.nch, st);
-    case 102: return launch_one<T, 1, 2, PRECISE, ZOH, false>(a, B, a.nch, st);
+    case 208: return launch_one<T, 2, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 108: return launch_one<T, 1, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 104: return launch_one<T, 1, 4, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 102: return launch_one<T, 1, 2, PRECISE, ZOH, 0>(a, B, a.nch, st);
     default: return cudaErrorInvalidValue;
   }
 }
@@ -444,25 +460,25 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
     const int shape = pick_thread_shape(c.B, c.d_inner, num_sms);
     return zoh ? launch_shape<T, PRECISE, true>(shape, a, c.B, st) : launch_shape<T, PRECISE, false>(shape, a, c.B, st);
   }
-  // chunked, two passes, 8 states per thread
+  // chunked, two launches, 8 states per thread.  Launch A: chunk 0 in full from the caller's state, chunks
+  // 1..n_end-1 state-only from zero; chain; launch B: chunks 1..nch-1 in full from their true initial states.
   const size_t n_state = (size_t)c.B * nch * c.d_inner * NST;
   float* h_end = chunk_ws;
   float* h_in = chunk_ws + n_state;
   float* sum_delta = chunk_ws + 2 * n_state;
   a.Lc = scan_chunk_len(c.L, nch); a.nch = nch;
   const int n_end = h_last ? nch : nch - 1;       // the last chunk's end state is only needed for h_last
-  ScanArgs p1 = a;
-  p1.h0 = nullptr; p1.h_last = h_end; p1.sum_delta = sum_delta; p1.z = nullptr; p1.y = nullptr;
-  cudaError_t e = zoh ? launch_one<T, 1, 8, PRECISE, true, true>(p1, c.B, n_end, st)
-                      : launch_one<T, 1, 8, PRECISE, false, true>(p1, c.B, n_end, st);
+  ScanArgs pa = a;
+  pa.h_last = h_end; pa.sum_delta = sum_delta; pa.chunk_off = 0;
+  cudaError_t e = zoh ? launch_one<T, 1, 8, PRECISE, true, 2>(pa, c.B, n_end, st) : launch_one<T, 1, 8, PRECISE, false, 2>(pa, c.B, n_end, st);
   if (e != cudaSuccess) return e;
   const long long n_thr = (long long)c.B * c.d_inner * NST;
-  chain_chunk_states<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(A, h0, h_end, sum_delta, h_in, h_last, c.B, c.d_inner, nch, n_end);
+  chain_chunk_states<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(A, h_end, sum_delta, h_in, h_last, c.B, c.d_inner, nch, n_end);
   count_launch();
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  a.h0 = h_in; a.h_last = nullptr;
-  return zoh ? launch_one<T, 1, 8, PRECISE, true, false>(a, c.B, nch, st) : launch_one<T, 1, 8, PRECISE, false, false>(a, c.B, nch, st);
+  a.h0 = h_in; a.h_last = nullptr; a.chunk_off = 1;
+  return zoh ? launch_one<T, 1, 8, PRECISE, true, 0>(a, c.B, nch - 1, st) : launch_one<T, 1, 8, PRECISE, false, 0>(a, c.B, nch - 1, st);
 }
 
 }  // namespace
@@ -478,7 +494,7 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, 
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, nullptr, gate_activated ? 1 : 0};
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, nullptr, gate_activated ? 1 : 0, 0};
   return c.dtype == ROM_BF16 ? launch_scan_t<__nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
                              : launch_scan_t<float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
 }
