@@ -229,11 +229,15 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
 
   // S3: grouped [Conv Proj | Gate Proj]
   // K = 1: the Gate Proj half is stored activated (SiLU); K > 1: raw, the activation follows the sum over slots in S4
-  Epilogue e_in{c.K == 1 ? EPI_INPROJ : EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, De, 0, nullptr, nullptr};
+  // Tensor path with one expert per token: the epilogue also puts every row back at its token's position, so the
+  // conv and the scan read H and the gate without indirection.
+  const bool in_token_order = tc && c.K == 1;
+  Epilogue e_in{c.K == 1 ? EPI_INPROJ : EPI_STORE, W + lay.XZp, 2 * De, nullptr, nullptr, nullptr, De, 0,
+                in_token_order ? reinterpret_cast<const int32_t*>(W + lay.assign_of_row) : nullptr, nullptr};
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
   ROM_STAGE_DONE();
   // S4: un-permute + sum over selected experts + conv + SiLU
-  ROM_CUDA(launch_conv(c, W + lay.XZp, row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
+  ROM_CUDA(launch_conv(c, W + lay.XZp, in_token_order ? nullptr : row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
   ROM_STAGE_DONE();
   // S5: x Proj -> delta_r | B | C
   Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N, nullptr, nullptr};
@@ -247,7 +251,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   // K = 1: the gate row of a token is its Gate Proj row in expert order; K > 1: the summed rows from S4
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;
   ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
-                       reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, c.K == 1 ? row_of_assign : nullptr,
+                       reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, (c.K == 1 && !in_token_order) ? row_of_assign : nullptr,
                        nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), true, st));
   ROM_STAGE_DONE();
   // S10 + S11.  Tensor path with one expert per token: the epilogue of the grouped Out Proj scales each row by

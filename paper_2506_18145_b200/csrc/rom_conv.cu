@@ -108,7 +108,7 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
       const int t = tb - 3 + r;
-      rix[r] = (t >= 0 && t < L) ? __ldg(row_of_assign + tok0 + t) : -1;
+      rix[r] = (t >= 0 && t < L) ? (row_of_assign ? __ldg(row_of_assign + tok0 + t) : (int32_t)(tok0 + t)) : -1;
     }
 #pragma unroll
     for (int r = 0; r < NR; ++r) {

@@ -302,10 +302,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool row_ok = row < M_valid;
       size_t out_row = (size_t)row;
       float scale = 1.0f;
-      if (MODE == EPI_OUTPROJ && row_ok) {
-        const int tok = __ldg(ep.row_token + row);
+      if ((MODE == EPI_OUTPROJ || (MODE == EPI_INPROJ && ep.row_token != nullptr)) && row_ok) {
+        const int tok = __ldg(ep.row_token + row);      // rows are written at their token's position
         row_ok = tok >= 0;
-        if (row_ok) { out_row = (size_t)tok; scale = __ldg(ep.row_scale + tok); }
+        if (row_ok) {
+          out_row = (size_t)tok;
+          if (MODE == EPI_OUTPROJ) scale = __ldg(ep.row_scale + tok);
+        }
       }
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * MAX_BLOCK_N;
       const int n_base = n_tile * block_n;

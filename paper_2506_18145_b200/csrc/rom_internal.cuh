@@ -64,7 +64,8 @@ enum EpiMode : int {
   EPI_STORE = 0,      // C[m, n] = acc                          (dtype)
   EPI_XPROJ = 1,      // n < R: delta_r[m, n] (dtype); then Bm[m, n-R], Cm[m, n-R-N] (fp32)
   EPI_SOFTPLUS = 2,   // Delta[m, n] = softplus(acc + bias[n])  (fp32)
-  EPI_INPROJ = 3,     // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype)
+  EPI_INPROJ = 3,     // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype); with row_token
+                      // (tensor path, top-1) row m is written at row row_token[m], i.e. back in token order
   EPI_OUTPROJ = 4     // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
                       // row_token[m] < 0 (segment padding) are skipped   (dtype; tensor path only)
 };
@@ -76,7 +77,7 @@ struct Epilogue {
   float* Cm;
   const float* bias;  // EPI_SOFTPLUS (may be null)
   int R, N;
-  const int32_t* row_token;   // EPI_OUTPROJ: token of each (padded) row, -1 in padding
+  const int32_t* row_token;   // EPI_OUTPROJ, EPI_INPROJ: token of each (padded) row, -1 in padding
   const float* row_scale;     // EPI_OUTPROJ: gate of each token
 };
 
@@ -97,6 +98,7 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
                            int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
                            const Epilogue& epi, int32_t* status, cudaStream_t st);
 
+// row_of_assign == nullptr (top-1, rows already in token order): row t of XZp belongs to token t.
 // Zs (K > 1 only): [T, d_inner], SiLU of the Gate Proj rows summed over the K slots.
 cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
                         const float* b_conv, void* U, void* Zs, cudaStream_t st);
