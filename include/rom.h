@@ -96,6 +96,16 @@ ROM_API int rom_route(const rom_config *cfg, const void *x, const void *W_r, con
               int32_t *topk_idx, float *gates, int32_t *counts, int32_t *offsets,
               int32_t *perm, int32_t *inv_perm, void *ws, size_t ws_bytes, void *stream);
 
+/* Load-balance statistic of the router of one layer (Appendix A.3, load balancing loss): runs the router
+ * (same logits, top-K and tie rule as rom_route) and returns
+ *   F[i]    = fraction of tokens dispatched to expert i = (assignments of i) / (B*L)   (sums to K),
+ *   Pbar[i] = mean over tokens of Softmax(X W_r)_i,
+ *   loss[0] = alpha * E * sum_i F[i] * Pbar[i]      (this layer's term; the paper uses alpha = 1e-3).
+ * F, Pbar [E] and loss [1] are fp32 device outputs; each may be NULL.  Sums over tokens are taken in a fixed
+ * order in fp64, so results are reproducible run to run.  Uses cfg->B, L, d_model, E, K, dtype.            */
+ROM_API int rom_route_balance(const rom_config *cfg, const void *x, const void *W_r, const float *b_r, float alpha,
+                      float *F, float *Pbar, float *loss, void *ws, size_t ws_bytes, void *stream);
+
 /* rom_route for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * is a deployment variant of the routing step above, with identical results.)
  *

@@ -21,7 +21,7 @@ ROM_OK = 0
 
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
-           "rom_num_stages", "rom_stage_name", "rom_route_noalloc")
+           "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance")
 
 
 class RomConfig(ctypes.Structure):
@@ -57,6 +57,7 @@ def lib() -> ctypes.CDLL:
         L.rom_workspace_size.argtypes = [cfgp, szp]
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
         L.rom_route_noalloc.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
+        L.rom_route_balance.argtypes = [cfgp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_scan.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_layer_forward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, i32p, vp, i32p, vp, ctypes.c_size_t, vp]
         L.rom_workspace_find.argtypes = [cfgp, ctypes.c_char_p, szp, szp]
@@ -140,6 +141,14 @@ def rom_route_noalloc(cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, 
                                  _ptr(offsets), _ptr(perm), _ptr(inv_perm), _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_route_noalloc")
+    return rc
+
+
+def rom_route_balance(cfg, x, W_r, b_r, alpha, F, Pbar, loss, ws, stream=None, check=True) -> int:
+    rc = lib().rom_route_balance(ctypes.byref(cfg), _ptr(x), _ptr(W_r), _ptr(b_r), ctypes.c_float(alpha), _ptr(F), _ptr(Pbar),
+                                 _ptr(loss), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_route_balance")
     return rc
 
 

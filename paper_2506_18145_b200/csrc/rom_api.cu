@@ -26,6 +26,7 @@ WsLayout make_layout(const rom_config& c) {
   l.num_m_tiles = take(sizeof(int32_t) * 4);
   l.tile_expert = take(sizeof(int32_t) * l.max_m_tiles);
   l.chunk_counts = take(sizeof(int32_t) * l.n_chunks * c.E);
+  l.chunk_prob = take(sizeof(double) * l.n_chunks * c.E);      // per-chunk softmax sums (rom_route_balance)
   l.topk_idx = take(sizeof(int32_t) * l.A);
   l.gates = take(sizeof(float) * l.A);
   l.perm = take(sizeof(int32_t) * l.A);
@@ -144,6 +145,20 @@ int rom_route(const rom_config* cfg, const void* x, const void* W_r, const float
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   LaunchCounter::count = 0;
   ROM_CUDA(launch_route(*cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm, static_cast<char*>(ws), lay, st));
+  return ROM_OK;
+}
+
+int rom_route_balance(const rom_config* cfg, const void* x, const void* W_r, const float* b_r, float alpha, float* F, float* Pbar,
+                      float* loss, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg, 1);
+  if (rc != ROM_OK) return rc;
+  if (!x || !W_r || !ws) return ROM_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_r) || !aligned16(ws)) return ROM_ERR_INVALID_ARG;
+  const WsLayout lay = make_layout(*cfg);
+  if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
+  if ((rc = check_device()) != ROM_OK) return rc;
+  LaunchCounter::count = 0;
+  ROM_CUDA(launch_balance(*cfg, x, W_r, b_r, alpha, F, Pbar, loss, static_cast<char*>(ws), lay, static_cast<cudaStream_t>(stream)));
   return ROM_OK;
 }
 

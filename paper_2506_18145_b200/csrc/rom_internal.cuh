@@ -47,7 +47,7 @@ inline size_t scan_ws_floats(int B, int De, int L) {
 
 // Workspace carving, identical for every entry point (host arithmetic only).
 struct WsLayout {
-  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts;
+  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts, chunk_prob;
   size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
   size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op, scan_ws;
   size_t total;
@@ -85,6 +85,14 @@ struct Epilogue {
 cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, const float* b_r,
                          int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
                          int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st);
+
+// launch_route with the per-chunk sums of the router softmax as an extra output (chunk_prob [n_chunks, E] fp64, or nullptr).
+cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W_r, const float* b_r,
+                               int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
+                               int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, double* chunk_prob, cudaStream_t st);
+// Router + load-balance statistic: F[E], Pbar[E], loss[1] (device fp32, each may be null).
+cudaError_t launch_balance(const rom_config& c, const void* x, const void* W_r, const float* b_r, float alpha,
+                           float* F, float* Pbar, float* loss, char* ws, const WsLayout& lay, cudaStream_t st);
 
 cudaError_t launch_gather_rows(const rom_config& c, const void* x, char* ws, const WsLayout& lay, cudaStream_t st);
 

@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(512)
 route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const float* __restrict__ b_r,
                   int T_tokens, int Dm, int E, int K, int gate_mode,
                   int32_t* __restrict__ topk_idx, float* __restrict__ gates,
-                  int32_t* __restrict__ chunk_counts) {
+                  int32_t* __restrict__ chunk_counts, double* __restrict__ chunk_prob) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int groups = (E + EG - 1) / EG;
   const int Epad = groups * EG;
@@ -138,10 +138,10 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
   if (tid < RT) {
     const int t = t0 + tid;
     const double* l = lg + tid * Epad;
+    double m = -INFINITY, denom = 1.0;
     if (t < T_tokens) {
-      double m = -INFINITY;
       for (int e = 0; e < E; ++e) { double v = l[e]; if (v > m) m = v; }   // NaN never raises m
-      double denom = 0.0;
+      denom = 0.0;
       for (int e = 0; e < E; ++e) denom += exp(l[e] - m);
       unsigned long long taken = 0ull;
       double gsel[kMaxK];
@@ -168,6 +168,16 @@ route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const floa
       }
     } else {
       for (int k = 0; k < K; ++k) idx_s[tid * K + k] = -1;
+    }
+    // optional: sum over the chunk's tokens of Softmax(X W_r), per expert (Appendix A.3 statistic); the lanes are
+    // added in a fixed shuffle order, so the result does not depend on scheduling
+    if (chunk_prob != nullptr) {
+      for (int e = 0; e < E; ++e) {
+        double pe = t < T_tokens ? exp(l[e] - m) / denom : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) pe += __shfl_down_sync(0xffffffffu, pe, o);
+        if (tid == 0) chunk_prob[(size_t)blockIdx.x * E + e] = pe;
+      }
     }
     // histogram of this chunk by warp ballots (warp 0 holds all 32 tokens)
     for (int e = 0; e < E; ++e) {
@@ -296,6 +306,46 @@ gather_rows(const uint4* __restrict__ x, uint4* __restrict__ x_perm, const int32
 cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, const float* b_r,
                          int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
                          int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st) {
+  return launch_route_stats(c, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm, ws, lay, nullptr, st);
+}
+
+// Load-balance statistic (Appendix A.3): F_i = assignments of expert i / tokens, Pbar_i = mean over tokens of
+// Softmax(X W_r)_i, loss = alpha * E * sum_i F_i * Pbar_i.  One block; chunk sums are added in chunk order.
+__global__ void __launch_bounds__(64)
+balance_finish(const double* __restrict__ chunk_prob, const int32_t* __restrict__ counts, int n_chunks, int E, int T_tokens,
+               float alpha, float* __restrict__ F, float* __restrict__ Pbar, float* __restrict__ loss) {
+  __shared__ double term[kMaxE];
+  const int e = threadIdx.x;
+  if (e < E) {
+    double ps = 0.0;
+    for (int c = 0; c < n_chunks; ++c) ps += chunk_prob[(size_t)c * E + e];
+    const double f = (double)counts[e] / (double)T_tokens, pb = ps / (double)T_tokens;
+    if (F) F[e] = (float)f;
+    if (Pbar) Pbar[e] = (float)pb;
+    term[e] = f * pb;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && loss) {
+    double sum = 0.0;
+    for (int i = 0; i < E; ++i) sum += term[i];
+    *loss = (float)((double)alpha * E * sum);
+  }
+}
+
+cudaError_t launch_balance(const rom_config& c, const void* x, const void* W_r, const float* b_r, float alpha,
+                           float* F, float* Pbar, float* loss, char* ws, const WsLayout& lay, cudaStream_t st) {
+  double* chunk_prob = reinterpret_cast<double*>(ws + lay.chunk_prob);
+  cudaError_t err = launch_route_stats(c, x, W_r, b_r, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, ws, lay, chunk_prob, st);
+  if (err != cudaSuccess) return err;
+  balance_finish<<<1, 64, 0, st>>>(chunk_prob, reinterpret_cast<const int32_t*>(ws + lay.counts), (int)lay.n_chunks, c.E, (int)lay.T,
+                                  alpha, F, Pbar, loss);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W_r, const float* b_r,
+                               int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
+                               int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, double* chunk_prob, cudaStream_t st) {
   const int T = (int)lay.T;
   const int groups = (c.E + EG - 1) / EG;
   const int Epad = groups * EG;
@@ -314,12 +364,12 @@ cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, co
     err = cudaFuncSetAttribute(route_logits_topk<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     route_logits_topk<__nv_bfloat16><<<blocks, threads, smem, st>>>(
-        (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts);
+        (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
   } else {
     err = cudaFuncSetAttribute(route_logits_topk<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     route_logits_topk<float><<<blocks, threads, smem, st>>>(
-        (const float*)x, (const float*)W_r, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts);
+        (const float*)x, (const float*)W_r, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
   }
   count_launch();
   route_offsets<<<1, 1024, 0, st>>>(chunk_counts, (int)lay.n_chunks, c.E,

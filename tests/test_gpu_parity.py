@@ -69,6 +69,25 @@ def test_route_bit_exact_full_size_configs(name):
         assert 4.5 < ratio < 5.5, ratio
 
 
+@pytest.mark.parametrize("kw", [dict(B=2, L=333, E=8, K=2), dict(B=1, L=50, E=5, K=1), dict(B=4, L=512, E=16, K=2, dtype="f32", router_bias_scale=2.0)])
+def test_route_balance_statistic(kw):
+    # Appendix A.3: F_i, mean softmax and alpha * E * sum F_i Pbar_i against the oracle on the same inputs
+    s = small_shape(**kw)
+    p = synth.make_inputs(s, recipe="unit")
+    cfg = rb.config_from_shape(s)
+    ws = rb.alloc_workspace(cfg)
+    F = torch.empty(s.E, dtype=torch.float32, device="cuda"); Pb = torch.empty_like(F); loss = torch.empty(1, dtype=torch.float32, device="cuda")
+    b_r = None if p["b_r"] is None else p["b_r"].cuda()
+    rb.rom_route_balance(cfg, p["x"].cuda(), p["W_r"].cuda(), b_r, 1e-3, F, Pb, loss, ws)
+    torch.cuda.synchronize()
+    idx, gate, P, logit = O.route(np64(p["x"]).reshape(s.T, s.d_model), np64(p["W_r"]), np64(p["b_r"]), s.K)
+    want, Fr = O.load_balance_loss(P, idx, alpha=1e-3)
+    np.testing.assert_allclose(F.cpu().numpy(), Fr, rtol=1e-6)
+    np.testing.assert_allclose(Pb.cpu().numpy(), P.mean(axis=0), rtol=2e-6)
+    np.testing.assert_allclose(float(loss.item()), want, rtol=2e-6)
+    assert abs(float(F.sum().item()) - s.K) < 1e-5
+
+
 # ---------------------------------------------------------------------------------------------- scan
 def run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed, use_ws=False):
     q = synth.make_scan_inputs(B, L, De, 16, dtype, seed, with_z=with_z, with_h0=with_h0)
