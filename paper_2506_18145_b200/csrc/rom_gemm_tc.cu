@@ -26,19 +26,27 @@
 namespace rom {
 namespace {
 
+constexpr int NUM_EPI_WARPS_C = 8;
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;            // 64 bf16 = 128 bytes = one swizzle row
 constexpr int MAX_BLOCK_N = 256;
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 4;
 constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;          // 16 KB
 constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;      // 32 KB
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int ACC_STAGES = 2;
 constexpr int TMEM_COLS = 512;
-constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_EPI_WARPS = NUM_EPI_WARPS_C;
 constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// Operand stages and epilogue staging per output op.  The softplus epilogue (dt Proj: only two K blocks per tile,
+// and the one GEMM here whose time is its fp32 output) gives up one operand stage for a 32 x 32 fp32 staging
+// square per epilogue warp, through which its stores become whole 128-byte row segments.
+__host__ __device__ constexpr int stages_of(int mode) { return mode == EPI_SOFTPLUS ? 3 : MAX_STAGES; }
+__host__ __device__ constexpr int out_stage_bytes_of(int mode) { return mode == EPI_SOFTPLUS ? NUM_EPI_WARPS_C * 32 * 32 * 4 : 0; }
+__host__ __device__ constexpr int smem_bytes_of(int mode) {
+  return stages_of(mode) * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
+}
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait polls before a wait gives up (a few seconds)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -176,12 +184,37 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
   }
 }
 
+// Softplus output op on a 32 (rows of this warp) x 32 (columns) accumulator square: every lane activates its row,
+// the square goes through a swizzled shared-memory staging area, and is written as whole 128-byte row segments
+// (8 lanes per row, 4 rows per store instruction) instead of 32 scattered 16-byte pieces.
+__device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, int row0, int M_valid, int n0, int N,
+                                               const uint32_t (&r)[32], const float4 (&bq)[8], int lane) {
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const float4 b = bq[c];
+    const float4 o = make_float4(softplus_fast(__uint_as_float(r[4 * c]) + b.x), softplus_fast(__uint_as_float(r[4 * c + 1]) + b.y),
+                                 softplus_fast(__uint_as_float(r[4 * c + 2]) + b.z), softplus_fast(__uint_as_float(r[4 * c + 3]) + b.w));
+    *reinterpret_cast<float4*>(sw + lane * 32 + ((c ^ (lane & 7)) << 2)) = o;
+  }
+  __syncwarp();
+  const int c = lane & 7;
+  const int n = n0 + 4 * c;
+#pragma unroll
+  for (int r4 = 0; r4 < 8; ++r4) {
+    const int R = r4 * 4 + (lane >> 3);
+    const float4 v = *reinterpret_cast<const float4*>(sw + R * 32 + ((c ^ (R & 7)) << 2));
+    if (row0 + R < M_valid && n < N) *reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.C) + (size_t)(row0 + R) * ep.ldc + n) = v;
+  }
+  __syncwarp();
+}
+
 template <int MODE>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M_max, int N, int Kd, int block_n, uint32_t idesc,
                const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ num_m_tiles_dev,
                Epilogue ep, int32_t* __restrict__ status) {
+  constexpr int STAGES = stages_of(MODE);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;               // 128B-swizzled tiles need 1024-byte alignment
@@ -193,6 +226,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + ACC_STAGES + a); };
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2 * ACC_STAGES));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  float* out_stage = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + 256);        // [8 warps][32][32] (softplus only)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -321,13 +355,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);     // in flight together with the tensor-memory load
         tmem_ld_wait(ra);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
-        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale, bq);
+        if (MODE == EPI_SOFTPLUS) epi_softplus32(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
+        else if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale, bq);
         ch += 2;
         if (ch >= n_chunks) break;
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);
         tmem_ld_wait(rb);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
-        if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale, bq);
+        if (MODE == EPI_SOFTPLUS) epi_softplus32(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
+        else if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale, bq);
         ch += 2;
       }
       tc_fence_before();
@@ -401,12 +437,13 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
               : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : epi.mode == EPI_OUTPROJ ? gemm_tc_kernel<EPI_OUTPROJ>
               : gemm_tc_kernel<EPI_SOFTPLUS>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  const int smem_bytes = smem_bytes_of(epi.mode);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   const int n_tiles = (N + block_n - 1) / block_n;
   const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
   const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
-  kern<<<grid, NUM_THREADS, SMEM_BYTES, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
+  kern<<<grid, NUM_THREADS, smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
   count_launch();
   return cudaGetLastError();
 }
