@@ -145,7 +145,8 @@ def run_reference(args, s):
     if rank != 0:
         return
     p = synth.make_inputs(s)
-    n_tok = min(s.L, 1024)
+    # bounded sample: about 64k oracle tokens (roughly a minute of host time) over the whole run
+    n_tok = min(s.L, max(64, min(1024, 65536 // max(args.steps, 1))))
     for _ in range(args.warmup):
         oracle_sample(s, p, min(n_tok, 256))
     times = []

@@ -84,7 +84,8 @@ ROM_API int rom_workspace_size(const rom_config *cfg, size_t *bytes);
 
 /* Router + top-K + dropless permutation (Section 4.2 routing equation; Section 5.1: no capacity
  * factor, no token dropping).
- *   logit[t,e] = b_r[e] + sum_d x[t,d] W_r[e,d], accumulated in fp64 in ascending d;
+ *   logit[t,e] = b_r[e] + sum_d x[t,d] W_r[e,d], accumulated in fp64 (exact products; the same summation order
+ *   for every expert, so equal weight rows give equal logits);
  *   P = softmax over all E; the K largest logits are selected, ties to the lowest expert id,
  *   slot k = k-th largest; gates per gate_mode.
  *   counts[e] = assignments of expert e; offsets = exclusive prefix sum (offsets[E] = T*K);
@@ -118,8 +119,10 @@ ROM_API int rom_route_balance(const rom_config *cfg, const void *x, const void *
  *
  * The caller passes inputs and outputs only; arguments, outputs and their meaning are those of
  * rom_route.  Limits: B*L <= 65536 tokens and B*L*K <= 131072 assignments (E <= 64, K <= 8 as
- * elsewhere); anything larger returns ROM_ERR_STATIC_SCRATCH and launches nothing -- use rom_route
- * with a caller-owned workspace instead.  The call itself allocates nothing, on the host or device.
+ * elsewhere), and the routing tables plus the fp64 copy of the router weights (8 * d_model * E bytes,
+ * E rounded up to 8) must fit the 3 MiB; anything larger returns ROM_ERR_STATIC_SCRATCH and launches
+ * nothing -- use rom_route with a caller-owned workspace instead.  The call itself allocates nothing,
+ * on the host or device.
  *
  * The first call on each GPU looks up the array's device address (once per device, with that
  * device current); make that first call before starting any stream capture.

@@ -26,6 +26,7 @@ WsLayout make_layout(const rom_config& c) {
   l.num_m_tiles = take(sizeof(int32_t) * 4);
   l.tile_expert = take(sizeof(int32_t) * l.max_m_tiles);
   l.chunk_counts = take(sizeof(int32_t) * l.n_chunks * c.E);
+  l.wr_f64 = take(sizeof(double) * (size_t)c.d_model * ((c.E + 7) / 8 * 8));   // router weights in fp64, experts padded to 8
   l.chunk_prob = take(sizeof(double) * l.n_chunks * c.E);      // per-chunk softmax sums (rom_route_balance)
   l.topk_idx = take(sizeof(int32_t) * l.A);
   l.gates = take(sizeof(float) * l.A);

@@ -47,7 +47,7 @@ inline size_t scan_ws_floats(int B, int De, int L) {
 
 // Workspace carving, identical for every entry point (host arithmetic only).
 struct WsLayout {
-  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts, chunk_prob;
+  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts, chunk_prob, wr_f64;
   size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
   size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op, scan_ws;
   size_t total;

@@ -2,9 +2,10 @@
 // factor and no token dropping), plus the row gather that feeds the grouped Conv/Gate projection.
 //
 // Kernels
-//   route_logits_topk : logits in fp64 (products of bf16 or fp32 inputs are exact in fp64 and the sum
-//                       runs strictly in ascending d, so the logits equal a left-to-right fp64 sum bit
-//                       for bit), softmax, top-K with ties to the lowest expert id, per-chunk histogram.
+//   route_weights_f64 : W_r in fp64, experts padded to a multiple of 8, once per call.
+//   route_logits_topk : logits in fp64 on the tensor cores (products of bf16 or fp32 inputs are exact in
+//                       fp64; every expert's sum is taken in the same order, so ties stay ties), softmax,
+//                       top-K with ties to the lowest expert id, per-chunk histogram.
 //   route_offsets     : per-expert exclusive scan of the chunk histograms (warp shuffles), expert
 //                       offsets, offsets padded to the GEMM row tile, row-tile -> expert map.
 //   route_scatter     : stable rank of every assignment inside its chunk by warp ballots; writes
@@ -15,124 +16,107 @@
 namespace rom {
 namespace {
 
-constexpr int RT = kChunkTokens;   // tokens per block of route_logits_topk = one routing chunk (lanes of a warp)
-constexpr int EG = 4;              // experts accumulated per thread (one warp = 32 tokens x EG experts)
-constexpr int DC = 64;             // d_model elements staged per step
+constexpr int RT = kChunkTokens;   // tokens per block of route_logits_topk = one routing chunk
+constexpr int NT8 = 8;             // experts per warp (one fp64 MMA column tile)
 
-template <typename T> struct XRow;
-template <> struct XRow<__nv_bfloat16> { static constexpr int kStrideBytes = DC * 2 + 16; };
-template <> struct XRow<float> { static constexpr int kStrideBytes = DC * 4 + 16; };
-
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, double (&xd)[8]) {
-  uint4 v = *reinterpret_cast<const uint4*>(p);
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    xd[2 * i] = (double)__uint_as_float(w[i] << 16);
-    xd[2 * i + 1] = (double)__uint_as_float(w[i] & 0xffff0000u);
-  }
-}
-__device__ __forceinline__ void load8(const float* p, double (&xd)[8]) {
-  float4 a = *reinterpret_cast<const float4*>(p);
-  float4 b = *reinterpret_cast<const float4*>(p + 4);
-  xd[0] = a.x; xd[1] = a.y; xd[2] = a.z; xd[3] = a.w;
-  xd[4] = b.x; xd[5] = b.y; xd[6] = b.z; xd[7] = b.w;
-}
-
-// One block = 32 tokens (one routing chunk).  Warp g accumulates experts [4g, 4g+4) for the 32 tokens
-// (lane = token): per element of d_model one x value from the lane's staged row and four router
-// weights broadcast from shared memory, four independent fp64 FMA chains, strictly ascending d.
+// Wd[e][d] = (double) W_r[e][d], experts padded with zero rows to a multiple of 8: the router weights in the
+// precision and layout the MMA fragments are loaded in (four consecutive d of one expert = 32 bytes).
 template <typename T>
-__global__ void __launch_bounds__(512)
-route_logits_topk(const T* __restrict__ x, const T* __restrict__ W_r, const float* __restrict__ b_r,
+__global__ void __launch_bounds__(256)
+route_weights_f64(const T* __restrict__ W_r, double* __restrict__ Wd, int Dm, int E, int Epad) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= Dm * Epad) return;
+  const int e = i / Dm;
+  Wd[i] = e < E ? (double)to_f32(W_r[i]) : 0.0;
+}
+
+// D (8x8) += A (8x4, row) * B (4x8, col), all fp64, on the tensor cores.  Lane l holds A[l/4][l%4], B[l%4][l/4]
+// and D[l/4][2*(l%4) + {0,1}].
+__device__ __forceinline__ void dmma_m8n8k4(double (&d)[2], double a, double b) {
+  asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+               : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
+}
+// four consecutive elements of a row as fp64
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, double (&xd)[4]) {
+  const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+  xd[0] = (double)__uint_as_float(v.x << 16); xd[1] = (double)__uint_as_float(v.x & 0xffff0000u);
+  xd[2] = (double)__uint_as_float(v.y << 16); xd[3] = (double)__uint_as_float(v.y & 0xffff0000u);
+}
+__device__ __forceinline__ void load4(const float* p, double (&xd)[4]) {
+  const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+  xd[0] = v.x; xd[1] = v.y; xd[2] = v.z; xd[3] = v.w;
+}
+
+// One block = 32 tokens (one routing chunk); warp w computes the logits of experts [8w, 8w+8) for them with
+// fp64 tensor-core MMAs (products of bf16/fp32 inputs are exact in fp64; every expert column is accumulated
+// in the same order, so equal weight rows give bit-equal logits and ties stay ties).  Per 16 elements of
+// d_model a lane reads 4 consecutive elements of one token row per 8-token tile (32-byte sectors, straight
+// from global memory) and 4 consecutive fp64 weights of one expert (L1/L2-resident copy); MMA j of the step
+// contracts elements {j, 4+j, 8+j, 12+j} of the 16.  No shared memory until the logits meet for the top-K.
+template <typename T>
+__global__ void __launch_bounds__(256)
+route_logits_topk(const T* __restrict__ x, const double* __restrict__ Wd, const float* __restrict__ b_r,
                   int T_tokens, int Dm, int E, int K, int gate_mode,
                   int32_t* __restrict__ topk_idx, float* __restrict__ gates,
                   int32_t* __restrict__ chunk_counts, double* __restrict__ chunk_prob) {
   extern __shared__ __align__(16) unsigned char smem[];
-  const int groups = (E + EG - 1) / EG;
-  const int Epad = groups * EG;
-  constexpr int XS = XRow<T>::kStrideBytes;
-  unsigned char* xs = smem;                                        // [2][RT][XS]   (double-buffered)
-  double* wsd = reinterpret_cast<double*>(smem + 2 * RT * XS);     // [2][groups][DC][EG]: a warp's four experts of one d are adjacent
-  double* lg = wsd + 2 * DC * Epad;                                // [RT][Epad]
+  const int Epad = (E + NT8 - 1) / NT8 * NT8;
+  double* lg = reinterpret_cast<double*>(smem);                    // [RT][Epad]
   int32_t* idx_s = reinterpret_cast<int32_t*>(lg + RT * Epad);     // [RT][K]
 
   const int tid = threadIdx.x;
-  const int tok = tid & 31;
-  const int g = tid >> 5;
+  const int lane = tid & 31, w = tid >> 5;
+  const int gq = lane >> 2, t4 = lane & 3;                        // fragment row / column group of this lane
   const int t0 = blockIdx.x * RT;
-  const int nthr = blockDim.x;
 
-  double acc[EG];
+  // accumulators: 4 tiles of 8 tokens x this warp's 8 experts; lane holds (token 8*mt + gq, experts 2*t4, 2*t4+1)
+  double acc[4][2];
 #pragma unroll
-  for (int e = 0; e < EG; ++e) {
-    const int ee = g * EG + e;
-    acc[e] = (b_r != nullptr && ee < E) ? (double)b_r[ee] : 0.0;
+  for (int mt = 0; mt < 4; ++mt) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int ee = w * NT8 + 2 * t4 + i;
+      acc[mt][i] = (b_r != nullptr && ee < E) ? (double)b_r[ee] : 0.0;
+    }
   }
-
-  // Chunk i+1 of x goes global -> shared with 16-byte asynchronous copies (rows past the end are
-  // zero-filled) and chunk i+1 of W_r is held in registers while chunk i is accumulated.
-  constexpr int VPR = DC * (int)sizeof(T) / 16;      // 16-byte vectors per row
-  constexpr int WPT = EG * DC / 32;                  // router weights per thread per chunk (Epad*DC / nthr)
-  auto copy_x = [&](int d0, int buf) {
-    for (int v = tid; v < RT * VPR; v += nthr) {
-      const int r = v / VPR, cv = v % VPR;
-      const bool in = t0 + r < T_tokens;
-      const unsigned char* src = reinterpret_cast<const unsigned char*>(x + (size_t)(in ? t0 + r : 0) * Dm + d0) + cv * 16;
-      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(xs + (buf * RT + r) * XS + cv * 16);
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(in ? 16 : 0) : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  };
-  float wpre[WPT];
-  auto fetch_w = [&](int d0) {
+  const T* xrow[4];
 #pragma unroll
-    for (int i = 0; i < WPT; ++i) {
-      const int v = tid + i * nthr, e = v / DC, d = v % DC;
-      wpre[i] = (e < E) ? to_f32(W_r[(size_t)e * Dm + d0 + d]) : 0.0f;
-    }
-  };
-  auto stash_w = [&](int buf) {
-#pragma unroll
-    for (int i = 0; i < WPT; ++i) {
-      const int v = tid + i * nthr, e = v / DC, d = v % DC;
-      wsd[((buf * groups + e / EG) * DC + d) * EG + (e % EG)] = (double)wpre[i];
-    }
-  };
+  for (int mt = 0; mt < 4; ++mt) xrow[mt] = x + (size_t)min(t0 + 8 * mt + gq, T_tokens - 1) * Dm + 4 * t4;   // rows past the end repeat the last token
+  const double* wrow = Wd + (size_t)(w * NT8 + gq) * Dm + 4 * t4;
 
-  copy_x(0, 0);
-  fetch_w(0);
-  stash_w(0);
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
-  __syncthreads();
-
-  int buf = 0;
-  for (int d0 = 0; d0 < Dm; d0 += DC, buf ^= 1) {
-    const bool more = d0 + DC < Dm;
-    if (more) { copy_x(d0 + DC, buf ^ 1); fetch_w(d0 + DC); }
-    const T* xrow = reinterpret_cast<const T*>(xs + (buf * RT + tok) * XS);
-    const double* wg = wsd + (buf * groups + g) * DC * EG;
-#pragma unroll 2
-    for (int d8 = 0; d8 < DC; d8 += 8) {
-      double xd[8];
-      load8(xrow + d8, xd);
+  double xa[4][4], wb[4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const double2 w01 = *reinterpret_cast<const double2*>(wg + (d8 + j) * EG);
-        const double2 w23 = *reinterpret_cast<const double2*>(wg + (d8 + j) * EG + 2);
-        acc[0] = fma(xd[j], w01.x, acc[0]);
-        acc[1] = fma(xd[j], w01.y, acc[1]);
-        acc[2] = fma(xd[j], w23.x, acc[2]);
-        acc[3] = fma(xd[j], w23.y, acc[3]);
-      }
-    }
-    if (more) stash_w(buf ^ 1);
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
+  for (int mt = 0; mt < 4; ++mt) load4(xrow[mt], xa[mt]);
+  {
+    const double2 b01 = __ldg(reinterpret_cast<const double2*>(wrow)), b23 = __ldg(reinterpret_cast<const double2*>(wrow) + 1);
+    wb[0] = b01.x; wb[1] = b01.y; wb[2] = b23.x; wb[3] = b23.y;
   }
-  __syncthreads();
+  for (int d0 = 0; d0 < Dm; d0 += 16) {
+    double xn[4][4], wn[4];
+    const int dn = d0 + 16 < Dm ? d0 + 16 : d0;                   // next step's operands in flight during this step's MMAs
 #pragma unroll
-  for (int e = 0; e < EG; ++e) lg[tok * Epad + g * EG + e] = acc[e];
+    for (int mt = 0; mt < 4; ++mt) load4(xrow[mt] + dn, xn[mt]);
+    {
+      const double2 b01 = __ldg(reinterpret_cast<const double2*>(wrow + dn)), b23 = __ldg(reinterpret_cast<const double2*>(wrow + dn) + 1);
+      wn[0] = b01.x; wn[1] = b01.y; wn[2] = b23.x; wn[3] = b23.y;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int mt = 0; mt < 4; ++mt) dmma_m8n8k4(acc[mt], xa[mt][j], wb[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      wb[j] = wn[j];
+#pragma unroll
+      for (int mt = 0; mt < 4; ++mt) xa[mt][j] = xn[mt][j];
+    }
+  }
+#pragma unroll
+  for (int mt = 0; mt < 4; ++mt) {
+    lg[(8 * mt + gq) * Epad + w * NT8 + 2 * t4] = acc[mt][0];
+    lg[(8 * mt + gq) * Epad + w * NT8 + 2 * t4 + 1] = acc[mt][1];
+  }
   __syncthreads();
 
   if (tid < RT) {
@@ -347,30 +331,29 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
                                int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
                                int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, double* chunk_prob, cudaStream_t st) {
   const int T = (int)lay.T;
-  const int groups = (c.E + EG - 1) / EG;
-  const int Epad = groups * EG;
   int32_t* idx_ws = topk_idx ? topk_idx : reinterpret_cast<int32_t*>(ws + lay.topk_idx);
   int32_t* chunk_counts = reinterpret_cast<int32_t*>(ws + lay.chunk_counts);
   int32_t* assign_of_row = reinterpret_cast<int32_t*>(ws + lay.assign_of_row);
   cudaError_t err = cudaMemsetAsync(assign_of_row, 0xff, sizeof(int32_t) * lay.rows_max, st);
   if (err != cudaSuccess) return err;
 
-  const int threads = RT * groups;
+  const int n_wtiles = (c.E + NT8 - 1) / NT8;
+  const int Epad8 = n_wtiles * NT8;
+  const int threads = 32 * n_wtiles;
   const int blocks = (T + RT - 1) / RT;
   const bool bf = c.dtype == ROM_BF16;
-  const size_t xs_bytes = (size_t)RT * (bf ? XRow<__nv_bfloat16>::kStrideBytes : XRow<float>::kStrideBytes);
-  const size_t smem = 2 * xs_bytes + sizeof(double) * (2 * (size_t)Epad * DC + (size_t)RT * Epad) + sizeof(int32_t) * RT * c.K;
-  if (bf) {
-    err = cudaFuncSetAttribute(route_logits_topk<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
+  double* Wd = reinterpret_cast<double*>(ws + lay.wr_f64);
+  const int nW = c.d_model * Epad8;
+  if (bf) route_weights_f64<__nv_bfloat16><<<(nW + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)W_r, Wd, c.d_model, c.E, Epad8);
+  else route_weights_f64<float><<<(nW + 255) / 256, 256, 0, st>>>((const float*)W_r, Wd, c.d_model, c.E, Epad8);
+  count_launch();
+  const size_t smem = sizeof(double) * (size_t)RT * Epad8 + sizeof(int32_t) * RT * c.K;
+  if (bf)
     route_logits_topk<__nv_bfloat16><<<blocks, threads, smem, st>>>(
-        (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
-  } else {
-    err = cudaFuncSetAttribute(route_logits_topk<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
+        (const __nv_bfloat16*)x, Wd, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
+  else
     route_logits_topk<float><<<blocks, threads, smem, st>>>(
-        (const float*)x, (const float*)W_r, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
-  }
+        (const float*)x, Wd, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
   count_launch();
   route_offsets<<<1, 1024, 0, st>>>(chunk_counts, (int)lay.n_chunks, c.E,
                                    reinterpret_cast<int32_t*>(ws + lay.counts), reinterpret_cast<int32_t*>(ws + lay.offsets),
