@@ -36,16 +36,21 @@ __device__ __forceinline__ void dmma_m8n8k4(double (&d)[2], double a, double b) 
   asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
                : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
 }
-// four consecutive elements of a row as fp64
-__device__ __forceinline__ void load4(const __nv_bfloat16* p, double (&xd)[4]) {
-  const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
-  xd[0] = (double)__uint_as_float(v.x << 16); xd[1] = (double)__uint_as_float(v.x & 0xffff0000u);
-  xd[2] = (double)__uint_as_float(v.y << 16); xd[3] = (double)__uint_as_float(v.y & 0xffff0000u);
-}
-__device__ __forceinline__ void load4(const float* p, double (&xd)[4]) {
-  const float4 v = __ldg(reinterpret_cast<const float4*>(p));
-  xd[0] = v.x; xd[1] = v.y; xd[2] = v.z; xd[3] = v.w;
-}
+// four consecutive elements of a row, kept as loaded and widened to fp64 when used
+template <typename T> struct RawX4;
+template <> struct RawX4<__nv_bfloat16> {
+  uint2 v;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { v = __ldg(reinterpret_cast<const uint2*>(p)); }
+  __device__ __forceinline__ void get(double (&xd)[4]) const {
+    xd[0] = (double)__uint_as_float(v.x << 16); xd[1] = (double)__uint_as_float(v.x & 0xffff0000u);
+    xd[2] = (double)__uint_as_float(v.y << 16); xd[3] = (double)__uint_as_float(v.y & 0xffff0000u);
+  }
+};
+template <> struct RawX4<float> {
+  float4 v;
+  __device__ __forceinline__ void load(const float* p) { v = __ldg(reinterpret_cast<const float4*>(p)); }
+  __device__ __forceinline__ void get(double (&xd)[4]) const { xd[0] = v.x; xd[1] = v.y; xd[2] = v.z; xd[3] = v.w; }
+};
 
 // One block = 32 tokens (one routing chunk); warp w computes the logits of experts [8w, 8w+8) for them with
 // fp64 tensor-core MMAs (products of bf16/fp32 inputs are exact in fp64; every expert column is accumulated
@@ -84,32 +89,33 @@ route_logits_topk(const T* __restrict__ x, const double* __restrict__ Wd, const 
   for (int mt = 0; mt < 4; ++mt) xrow[mt] = x + (size_t)min(t0 + 8 * mt + gq, T_tokens - 1) * Dm + 4 * t4;   // rows past the end repeat the last token
   const double* wrow = Wd + (size_t)(w * NT8 + gq) * Dm + 4 * t4;
 
-  double xa[4][4], wb[4];
+  // operands of the next PF-1 steps are in flight (raw, unconverted) while one step is contracted
+  // (d_model is a multiple of 64, so there are at least PF steps)
+  constexpr int PF = 4;
+  RawX4<T> rx[PF][4];
+  double2 rw[PF][2];
+  auto fetch = [&](int d, RawX4<T> (&xo)[4], double2 (&wo)[2]) {
 #pragma unroll
-  for (int mt = 0; mt < 4; ++mt) load4(xrow[mt], xa[mt]);
-  {
-    const double2 b01 = __ldg(reinterpret_cast<const double2*>(wrow)), b23 = __ldg(reinterpret_cast<const double2*>(wrow) + 1);
-    wb[0] = b01.x; wb[1] = b01.y; wb[2] = b23.x; wb[3] = b23.y;
-  }
-  for (int d0 = 0; d0 < Dm; d0 += 16) {
-    double xn[4][4], wn[4];
-    const int dn = d0 + 16 < Dm ? d0 + 16 : d0;                   // next step's operands in flight during this step's MMAs
+    for (int mt = 0; mt < 4; ++mt) xo[mt].load(xrow[mt] + d);
+    wo[0] = __ldg(reinterpret_cast<const double2*>(wrow + d));
+    wo[1] = __ldg(reinterpret_cast<const double2*>(wrow + d) + 1);
+  };
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt) load4(xrow[mt] + dn, xn[mt]);
-    {
-      const double2 b01 = __ldg(reinterpret_cast<const double2*>(wrow + dn)), b23 = __ldg(reinterpret_cast<const double2*>(wrow + dn) + 1);
-      wn[0] = b01.x; wn[1] = b01.y; wn[2] = b23.x; wn[3] = b23.y;
-    }
+  for (int i = 0; i < PF - 1; ++i) fetch(16 * i, rx[i], rw[i]);
+  for (int d0 = 0; d0 < Dm; d0 += 16 * PF) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int i = 0; i < PF; ++i) {
+      const int dn = d0 + 16 * (i + PF - 1);                              // step that enters the ring now
+      if (dn < Dm) fetch(dn, rx[(i + PF - 1) % PF], rw[(i + PF - 1) % PF]);
+      const double wb[4] = {rw[i][0].x, rw[i][0].y, rw[i][1].x, rw[i][1].y};
+      double xa[4][4];
 #pragma unroll
-      for (int mt = 0; mt < 4; ++mt) dmma_m8n8k4(acc[mt], xa[mt][j], wb[j]);
-    }
+      for (int mt = 0; mt < 4; ++mt) rx[i][mt].get(xa[mt]);
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      wb[j] = wn[j];
+      for (int j = 0; j < 4; ++j) {
 #pragma unroll
-      for (int mt = 0; mt < 4; ++mt) xa[mt][j] = xn[mt][j];
+        for (int mt = 0; mt < 4; ++mt) dmma_m8n8k4(acc[mt], xa[mt][j], wb[j]);
+      }
     }
   }
 #pragma unroll
@@ -184,17 +190,27 @@ route_offsets(int32_t* __restrict__ chunk_counts, int n_chunks, int E,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   for (int e = warp; e < E; e += nwarps) {
     int carry = 0;
-    for (int c0 = 0; c0 < n_chunks; c0 += 32) {
-      const int c = c0 + lane;
-      const int v = (c < n_chunks) ? chunk_counts[(size_t)c * E + e] : 0;
-      int inc = v;
+    constexpr int UB = 8;                         // chunks-of-32 whose loads are issued together
+    for (int cb = 0; cb < n_chunks; cb += 32 * UB) {
+      int vv[UB];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int n = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += n;
+      for (int i = 0; i < UB; ++i) {
+        const int c = cb + 32 * i + lane;
+        vv[i] = (c < n_chunks) ? chunk_counts[(size_t)c * E + e] : 0;
       }
-      if (c < n_chunks) chunk_counts[(size_t)c * E + e] = carry + inc - v;    // exclusive base
-      carry += __shfl_sync(0xffffffffu, inc, 31);
+#pragma unroll
+      for (int i = 0; i < UB; ++i) {
+        const int c = cb + 32 * i + lane;
+        const int v = vv[i];
+        int inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          int n = __shfl_up_sync(0xffffffffu, inc, o);
+          if (lane >= o) inc += n;
+        }
+        if (c < n_chunks) chunk_counts[(size_t)c * E + e] = carry + inc - v;    // exclusive base
+        carry += __shfl_sync(0xffffffffu, inc, 31);
+      }
     }
     if (lane == 0) cnt[e] = carry;
   }
