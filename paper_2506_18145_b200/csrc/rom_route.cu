@@ -59,18 +59,22 @@ template <> struct RawX4<float> {
 // from global memory) and 4 consecutive fp64 weights of one expert (L1/L2-resident copy); MMA j of the step
 // contracts elements {j, 4+j, 8+j, 12+j} of the 16.  No shared memory until the logits meet for the top-K.
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 route_logits_topk(const T* __restrict__ x, const double* __restrict__ Wd, const float* __restrict__ b_r,
                   int T_tokens, int Dm, int E, int K, int gate_mode,
                   int32_t* __restrict__ topk_idx, float* __restrict__ gates,
                   int32_t* __restrict__ chunk_counts, double* __restrict__ chunk_prob) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int Epad = (E + NT8 - 1) / NT8 * NT8;
-  double* lg = reinterpret_cast<double*>(smem);                    // [RT][Epad]
-  int32_t* idx_s = reinterpret_cast<int32_t*>(lg + RT * Epad);     // [RT][K]
+  const int n_wtiles = Epad / NT8;
+  const int dsplit = (blockDim.x >> 5) / n_wtiles;                 // warps that share one expert tile, each on its own d range
+  double* lg = reinterpret_cast<double*>(smem);                    // [dsplit][RT][Epad] partial logits; [0] becomes the sum
+  int32_t* idx_s = reinterpret_cast<int32_t*>(lg + dsplit * RT * Epad);   // [RT][K]
 
   const int tid = threadIdx.x;
-  const int lane = tid & 31, w = tid >> 5;
+  const int lane = tid & 31, wq = tid >> 5;
+  const int w = wq / dsplit, dq = wq % dsplit;                     // expert tile, d range [dq, dq+1) * Dm / dsplit
+  const int d_lo = (Dm / 16 * dq / dsplit) * 16, d_hi = (Dm / 16 * (dq + 1) / dsplit) * 16;
   const int gq = lane >> 2, t4 = lane & 3;                        // fragment row / column group of this lane
   const int t0 = blockIdx.x * RT;
 
@@ -81,7 +85,7 @@ route_logits_topk(const T* __restrict__ x, const double* __restrict__ Wd, const 
 #pragma unroll
     for (int i = 0; i < 2; ++i) {
       const int ee = w * NT8 + 2 * t4 + i;
-      acc[mt][i] = (b_r != nullptr && ee < E) ? (double)b_r[ee] : 0.0;
+      acc[mt][i] = (b_r != nullptr && ee < E && dq == 0) ? (double)b_r[ee] : 0.0;
     }
   }
   const T* xrow[4];
@@ -101,12 +105,14 @@ route_logits_topk(const T* __restrict__ x, const double* __restrict__ Wd, const 
     wo[1] = __ldg(reinterpret_cast<const double2*>(wrow + d) + 1);
   };
 #pragma unroll
-  for (int i = 0; i < PF - 1; ++i) fetch(16 * i, rx[i], rw[i]);
-  for (int d0 = 0; d0 < Dm; d0 += 16 * PF) {
+  for (int i = 0; i < PF - 1; ++i)
+    if (d_lo + 16 * i < d_hi) fetch(d_lo + 16 * i, rx[i], rw[i]);
+  for (int d0 = d_lo; d0 < d_hi; d0 += 16 * PF) {
 #pragma unroll
     for (int i = 0; i < PF; ++i) {
+      if (d0 + 16 * i >= d_hi) break;
       const int dn = d0 + 16 * (i + PF - 1);                              // step that enters the ring now
-      if (dn < Dm) fetch(dn, rx[(i + PF - 1) % PF], rw[(i + PF - 1) % PF]);
+      if (dn < d_hi) fetch(dn, rx[(i + PF - 1) % PF], rw[(i + PF - 1) % PF]);
       const double wb[4] = {rw[i][0].x, rw[i][0].y, rw[i][1].x, rw[i][1].y};
       double xa[4][4];
 #pragma unroll
@@ -120,8 +126,16 @@ route_logits_topk(const T* __restrict__ x, const double* __restrict__ Wd, const 
   }
 #pragma unroll
   for (int mt = 0; mt < 4; ++mt) {
-    lg[(8 * mt + gq) * Epad + w * NT8 + 2 * t4] = acc[mt][0];
-    lg[(8 * mt + gq) * Epad + w * NT8 + 2 * t4 + 1] = acc[mt][1];
+    lg[(dq * RT + 8 * mt + gq) * Epad + w * NT8 + 2 * t4] = acc[mt][0];
+    lg[(dq * RT + 8 * mt + gq) * Epad + w * NT8 + 2 * t4 + 1] = acc[mt][1];
+  }
+  __syncthreads();
+
+  // the d ranges are added in a fixed order, the same for every expert
+  for (int i = tid; i < RT * Epad; i += blockDim.x) {
+    double v = lg[i];
+    for (int q = 1; q < dsplit; ++q) v += lg[q * RT * Epad + i];
+    lg[i] = v;
   }
   __syncthreads();
 
@@ -355,7 +369,10 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
 
   const int n_wtiles = (c.E + NT8 - 1) / NT8;
   const int Epad8 = n_wtiles * NT8;
-  const int threads = 32 * n_wtiles;
+  // warps per chunk: one per 8-expert tile, times a split of d_model (up to 4 ranges) that puts more loads in flight
+  int dsplit = 4;
+  while (dsplit > 1 && (n_wtiles * dsplit > 16 || c.d_model / 16 < 4 * dsplit)) dsplit >>= 1;
+  const int threads = 32 * n_wtiles * dsplit;
   const int blocks = (T + RT - 1) / RT;
   const bool bf = c.dtype == ROM_BF16;
   double* Wd = reinterpret_cast<double*>(ws + lay.wr_f64);
@@ -363,7 +380,7 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
   if (bf) route_weights_f64<__nv_bfloat16><<<(nW + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)W_r, Wd, c.d_model, c.E, Epad8);
   else route_weights_f64<float><<<(nW + 255) / 256, 256, 0, st>>>((const float*)W_r, Wd, c.d_model, c.E, Epad8);
   count_launch();
-  const size_t smem = sizeof(double) * (size_t)RT * Epad8 + sizeof(int32_t) * RT * c.K;
+  const size_t smem = sizeof(double) * (size_t)dsplit * RT * Epad8 + sizeof(int32_t) * RT * c.K;
   if (bf)
     route_logits_topk<__nv_bfloat16><<<blocks, threads, smem, st>>>(
         (const __nv_bfloat16*)x, Wd, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
