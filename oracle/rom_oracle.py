@@ -23,12 +23,16 @@ Readings taken where the paper is silent (each is a flag or an optional argument
   * disc_mode 0 = zero-order hold exactly as printed (diagonal A);
     disc_mode 1 = B-bar = Delta * B.
   * D skip, conv bias, dt bias, router bias are optional (None = paper-literal).
+  * per-expert x Proj / dt Proj (an ablation row of Section 5.3, no equation printed):
+    indicator-only sums like H_t; each expert's delta passes through its own dt Proj.
 
 Pins (tests/test_oracle_pins.py): dense-Mamba reduction (E=K=1), brute-force
 unrolled SSM, K=E uniform gates = mean of experts, batch-permutation invariance,
 identical experts, geometric-series closed form, exact ODE solution for ZOH,
 identity conv tap + causality, permutation tables vs brute force and a stable
-sort, gate sums, tie rule, two-half scan, parameter counts printed in the paper.
+sort, gate sums, tie rule, two-half scan, parameter counts printed in the paper;
+per-expert small projections: E=1 / identical experts reduce to the shared form, rows of
+one expert equal the shared form with that expert's matrices, per-token brute force.
 """
 from __future__ import annotations
 
@@ -208,6 +212,40 @@ def small_proj(U, W_x, W_dt, b_dt, dt_rank, d_state):
     return delta, Bm, Cm, softplus(pre)
 
 
+def small_proj_routed(U, W_x, W_dt, b_dt, idx, dt_rank, d_state):
+    """x Proj and dt Proj as per-expert layers under the shared routing decision: the ablation
+    "RoM (Conv, Gate, dt, x, Out)" of Section 5.3 (Section 4.3 shares them by default).  The paper
+    prints no equation for this variant; it is read in the pattern of the equations for H_t and G
+    (indicator-only sums over the selected experts):
+        (delta_i, B_i, C_i) = U_t W_x,i ,  B_t = sum_i 1_i B_i ,  C_t = sum_i 1_i C_i ,
+        Delta_t = softplus( sum_i 1_i delta_i W_dt,i + b_dt ),
+    each expert's delta_i going through that expert's own dt Proj; b_dt stays shared.
+    U[T,D_e]; W_x[E, R+2N, D_e]; W_dt[E, D_e, R]; idx[T,K].  Returns Bm[T,N], Cm[T,N], Delta[T,D_e].
+    """
+    U = np.asarray(U, dtype=F64)
+    W_x = np.asarray(W_x, dtype=F64)
+    W_dt = np.asarray(W_dt, dtype=F64)
+    R, N = dt_rank, d_state
+    T, De = U.shape
+    E = W_x.shape[0]
+    Bm = np.zeros((T, N), dtype=F64)
+    Cm = np.zeros((T, N), dtype=F64)
+    pre = np.zeros((T, De), dtype=F64)
+    K = idx.shape[1]
+    for k in range(K):
+        for e in range(E):
+            tok = np.nonzero(idx[:, k] == e)[0]
+            if tok.size == 0:
+                continue
+            xdbl = U[tok] @ W_x[e].T
+            Bm[tok] += xdbl[:, R:R + N]
+            Cm[tok] += xdbl[:, R + N:R + 2 * N]
+            pre[tok] += xdbl[:, :R] @ W_dt[e].T
+    if b_dt is not None:
+        pre = pre + np.asarray(b_dt, dtype=F64)[None, :]
+    return Bm, Cm, softplus(pre)
+
+
 # --------------------------------------------------------------------------- S7 selective scan
 def selective_scan(U, Delta, A, Bm, Cm, D=None, h0=None, disc_mode=0):
     """Linear recurrence of Section 3.1:  h_t = A-bar h_{t-1} + B-bar U_t,  Y_t = C h_t
@@ -272,6 +310,8 @@ def expert_out_proj(Yg, W_out, idx, gate):
 def rom_layer_forward(x, W_r, b_r, W_inz, w_conv, b_conv, W_x, W_dt, b_dt, A, D, W_out,
                       K, dt_rank, gate_mode=0, disc_mode=0, return_intermediates=False):
     """Forward pass of one RoM layer (Section 4.2 with the shared small layers of 4.3).
+    W_x[R+2N, D_e] and W_dt[D_e, R] are the shared x Proj / dt Proj; three-dimensional
+    W_x[E, ...], W_dt[E, ...] select the per-expert variant (small_proj_routed).
 
     x[B,L,D_m].  Returns out[B,L,D_m] (and a dict of every intermediate if asked).
     """
@@ -287,7 +327,11 @@ def rom_layer_forward(x, W_r, b_r, W_inz, w_conv, b_conv, W_x, W_dt, b_dt, A, D,
     H, Zpre = expert_in_proj(xt, W_inz, idx)
     De = H.shape[1]
     U = conv_silu(H.reshape(Bsz, L, De), w_conv, b_conv)
-    delta, Bm, Cm, Delta = small_proj(U.reshape(T, De), W_x, W_dt, b_dt, dt_rank, N)
+    if np.asarray(W_x).ndim == 3:          # per-expert x Proj / dt Proj (ablation of Section 5.3)
+        delta = None
+        Bm, Cm, Delta = small_proj_routed(U.reshape(T, De), W_x, W_dt, b_dt, idx, dt_rank, N)
+    else:
+        delta, Bm, Cm, Delta = small_proj(U.reshape(T, De), W_x, W_dt, b_dt, dt_rank, N)
     Y, h_last = selective_scan(U, Delta.reshape(Bsz, L, De), A, Bm.reshape(Bsz, L, N),
                                Cm.reshape(Bsz, L, N), D, None, disc_mode)
     Yg = gated(Y.reshape(T, De), Zpre)

@@ -355,6 +355,79 @@ def test_small_proj_split_and_softplus_vs_library():
     np.testing.assert_allclose(O.softplus(np.array([-800.0, 0.0, 800.0])), [0.0, math.log(2.0), 800.0], atol=1e-300)
 
 
+# ---------------------------------------------------------------------------------------------- per-expert x Proj / dt Proj
+def _routed_small_case(seed, T=23, De=6, R=3, N=4, E=4, K=2):
+    g = rng(seed)
+    U = g.normal(size=(T, De)); W_x = g.normal(size=(E, R + 2 * N, De)); W_dt = g.normal(size=(E, De, R))
+    b = g.normal(size=De)
+    idx = np.stack([g.permutation(E)[:K] for _ in range(T)]).astype(np.int32)
+    return U, W_x, W_dt, b, idx
+
+
+def test_routed_small_proj_vs_per_token_loop():
+    """Brute force per token with scalar loops: B_t, C_t are indicator sums of the selected experts' rows of
+    U_t W_x,i and the softplus argument sums each expert's delta through its own dt Proj."""
+    T, De, R, N, E, K = 23, 6, 3, 4, 4, 2
+    U, W_x, W_dt, b, idx = _routed_small_case(21, T, De, R, N, E, K)
+    Bm, Cm, Dl = O.small_proj_routed(U, W_x, W_dt, b, idx, R, N)
+    for t in range(T):
+        for n in range(N):
+            assert abs(Bm[t, n] - sum(sum(W_x[idx[t, k], R + n, c] * U[t, c] for c in range(De)) for k in range(K))) < 1e-12
+            assert abs(Cm[t, n] - sum(sum(W_x[idx[t, k], R + N + n, c] * U[t, c] for c in range(De)) for k in range(K))) < 1e-12
+        for c in range(De):
+            pre = b[c]
+            for k in range(K):
+                e = idx[t, k]
+                for r in range(R):
+                    pre += W_dt[e, c, r] * sum(W_x[e, r, cc] * U[t, cc] for cc in range(De))
+            assert abs(Dl[t, c] - float(F.softplus(torch.tensor(pre, dtype=torch.float64)))) < 1e-12
+
+
+def test_routed_small_proj_rows_of_one_expert_equal_the_shared_form():
+    """Top-1: the tokens of expert e get exactly what the shared x Proj / dt Proj computes with that expert's
+    matrices; E = 1 and identical experts reduce to the shared form (K identical experts: K-fold sums)."""
+    T, De, R, N, E = 40, 6, 3, 4, 4
+    U, W_x, W_dt, b, idx2 = _routed_small_case(22, T, De, R, N, E, 2)
+    idx = idx2[:, :1]
+    Bm, Cm, Dl = O.small_proj_routed(U, W_x, W_dt, b, idx, R, N)
+    seen = 0
+    for e in range(E):
+        tok = np.nonzero(idx[:, 0] == e)[0]
+        seen += tok.size
+        _, Be, Ce, De_ = O.small_proj(U, W_x[e], W_dt[e], b, R, N)
+        np.testing.assert_allclose(Bm[tok], Be[tok], rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(Cm[tok], Ce[tok], rtol=1e-12, atol=1e-13)
+        np.testing.assert_allclose(Dl[tok], De_[tok], rtol=1e-12, atol=1e-13)
+    assert seen == T
+    # identical experts, K = 2: delta, B and C all double (the shared form with 2 W_x)
+    Wx_same = np.repeat(W_x[:1], E, axis=0); Wdt_same = np.repeat(W_dt[:1], E, axis=0)
+    B2, C2, D2 = O.small_proj_routed(U, Wx_same, Wdt_same, b, idx2, R, N)
+    _, Bs, Cs, Ds = O.small_proj(U, 2.0 * W_x[0], W_dt[0], b, R, N)
+    np.testing.assert_allclose(B2, Bs, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(C2, Cs, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(D2, Ds, rtol=1e-12, atol=1e-13)
+
+
+def test_layer_with_identical_small_experts_equals_shared_layer():
+    """Whole layer: stacking E copies of the shared x Proj / dt Proj as per-expert matrices changes nothing at
+    top-1; with E = 1 the per-expert layer is the dense Mamba layer."""
+    p, s = small_layer(23, E=3)
+    shared = run_layer(p, K=1, R=s["R"])
+    q = dict(p)
+    q["W_x"] = np.repeat(p["W_x"][None], s["E"], axis=0); q["W_dt"] = np.repeat(p["W_dt"][None], s["E"], axis=0)
+    np.testing.assert_allclose(run_layer(q, K=1, R=s["R"]), shared, rtol=1e-12, atol=1e-14)
+    # distinct small experts do change the output (the mode is not a no-op)
+    g = rng(24)
+    q["W_x"] = q["W_x"] + 0.3 * g.normal(size=q["W_x"].shape)
+    assert np.abs(run_layer(q, K=1, R=s["R"]) - shared).max() > 1e-3
+    p1, s1 = small_layer(25, E=1)
+    De = s1["De"]
+    q1 = dict(p1); q1["W_x"] = p1["W_x"][None]; q1["W_dt"] = p1["W_dt"][None]
+    ref = dense_mamba_torch(p1["x"], p1["W_inz"][0, :De], p1["W_inz"][0, De:], p1["w_conv"], p1["b_conv"],
+                            p1["W_x"], p1["W_dt"], p1["b_dt"], p1["A"], p1["D"], p1["W_out"][0], s1["R"])
+    np.testing.assert_allclose(run_layer(q1, K=1, R=s1["R"]), ref, rtol=1e-10, atol=1e-12)
+
+
 # ---------------------------------------------------------------------------------------------- P11
 def test_wiring_reproduces_paper_parameter_counts():
     rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_param_counts.txt")) if l.strip() and not l.startswith("#")]
