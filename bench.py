@@ -144,7 +144,7 @@ def run_reference(args, s):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    p = synth.make_inputs(s)
+    p = synth.make_inputs(s, routed_small=args.small_proj == "routed")
     # bounded sample: about 64k oracle tokens (roughly a minute of host time) over the whole run
     n_tok = min(s.L, max(64, min(1024, 65536 // max(args.steps, 1))))
     for _ in range(args.warmup):
@@ -160,7 +160,7 @@ def run_reference(args, s):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(s),
+            "config": workload_config(s, args.small_proj),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -214,8 +214,8 @@ def run_stage(args, s):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(s):
-    return {"workload": s.name, "B": s.B, "L": s.L, "d_model": s.d_model, "d_inner": s.d_inner, "d_state": s.d_state,
+def workload_config(s, small_proj="shared"):
+    return {"workload": s.name, "small_proj": small_proj, "B": s.B, "L": s.L, "d_model": s.d_model, "d_inner": s.d_inner, "d_state": s.d_state,
             "d_conv": s.d_conv, "dt_rank": s.dt_rank, "E": s.E, "K": s.K, "storage": s.dtype,
             "l2": "inputs+weights larger than L2 (no flush between iterations)"}
 
@@ -229,6 +229,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="run the projections on the fp32-FMA bisecting path")
+    ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
+                    help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
+                         "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
     ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route"],
                     help="layer: the whole forward (the benchmark); scan / route: that entry point alone, timed in isolation "
                          "at the workload's shape (kernel studies and ncu captures; prints a short JSON line)")
@@ -258,9 +261,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
 
-    p = synth.make_inputs(s)
+    routed_small = args.small_proj == "routed"
+    p = synth.make_inputs(s, routed_small=routed_small)
     d = {k: (None if v is None else v.to(dev)) for k, v in p.items()}
-    cfg = rb.config_from_shape(s, flags=rb.ROM_FLAG_SIMT_GEMM if args.simt else 0)
+    cfg = rb.config_from_shape(s, flags=rb.ROM_FLAG_SIMT_GEMM if args.simt else 0, small_proj_experts=s.E if routed_small else 0)
     weights = rb.make_weights(d)
     ws = rb.alloc_workspace(cfg, dev)
     x_dev = d["x"]
@@ -372,7 +376,7 @@ def main():
         line = {"metric": METRIC, "value": replicas.job_throughput(s.T, world, args.steps, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if s.dtype == "bf16" else "f32", "data": "synthetic",
-                "config": workload_config(s), "clocks": clocks,
+                "config": workload_config(s, args.small_proj), "clocks": clocks,
                 "e2e": {"value": replicas.job_throughput(s.T, world, args.steps, ms_e2e), "unit": UNIT,
                         "h2d_bytes_per_step": x_host.numel() * x_host.element_size(),
                         "d2h_bytes_per_step": out_host.numel() * out_host.element_size()},

@@ -58,7 +58,9 @@ typedef struct {
                                  1: P_i renormalised over the selected K (the sentence above it)   */
   int32_t disc_mode;          /* 0: zero-order hold B-bar (Section 3.1); 1: B-bar = Delta * B      */
   int32_t flags;              /* ROM_FLAG_* bits                                                  */
-  int32_t reserved;           /* must be 0                                                        */
+  int32_t small_proj_experts; /* 0 or 1: x Proj / dt Proj shared by all experts (Section 4.3, the method as
+                                 proposed); E: one x Proj / dt Proj per expert under the same routing
+                                 decision (the "(Conv, Gate, dt, x, Out)" ablation row of Section 5.3)      */
 } rom_config;
 
 #define ROM_FLAG_SIMT_GEMM 1  /* run every projection on the plain fp32-FMA kernels (bisecting aid;
@@ -71,8 +73,10 @@ typedef struct {                /* all read-only device pointers                
                                                                     rows [D_e,2D_e): Gate Proj W_g,i^T */
   const void  *w_conv;          /* [d_conv, d_inner]         dtype  tap d_conv-1 = current token   */
   const float *b_conv;          /* [d_inner] or NULL                                              */
-  const void  *W_x;             /* [dt_rank+2*d_state, d_inner] dtype  rows delta | B | C (shared) */
-  const void  *W_dt;            /* [d_inner, dt_rank]        dtype  (shared)                       */
+  const void  *W_x;             /* [dt_rank+2*d_state, d_inner] dtype  rows delta | B | C (shared);
+                                   [E, dt_rank+2*d_state, d_inner] when small_proj_experts == E      */
+  const void  *W_dt;            /* [d_inner, dt_rank]        dtype  (shared); [E, d_inner, dt_rank]
+                                   when small_proj_experts == E                                      */
   const float *b_dt;            /* [d_inner] or NULL                                              */
   const float *A;               /* [d_inner, d_state]        fp32, strictly negative              */
   const float *D;               /* [d_inner] or NULL         skip (not in the paper's equations)   */
@@ -152,7 +156,12 @@ ROM_API int rom_scan(const rom_config *cfg, const void *u, const float *delta, c
  *   softplus -> selective scan -> * SiLU(gate) -> re-permute with the same routing -> per-expert
  *   Out Proj -> gate-weighted sum over the selected experts.
  *   x, out : [B, L, d_model] dtype.  topk_idx_out [T,K] i32, gates_out [T,K] f32, counts_out [E] i32
- *   may each be NULL.                                                                             */
+ *   may each be NULL.
+ * With cfg->small_proj_experts == E the x Proj and dt Proj are per-expert layers under the same
+ * routing (the paper prints no equation for this ablation; it is taken in the pattern of H_t and G):
+ *   (delta_i, B_i, C_i) = U_t W_x,i;  B_t = sum_i 1_i B_i;  C_t = sum_i 1_i C_i;
+ *   Delta_t = softplus(sum_i 1_i delta_i W_dt,i + b_dt)  -- indicator-only sums over the selected
+ *   experts in ascending slot order, each expert's delta_i through its own dt Proj, b_dt shared.   */
 ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const void *x, void *out,
                       int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
                       void *ws, size_t ws_bytes, void *stream);

@@ -27,7 +27,7 @@ EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "
 class RomConfig(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "L", "d_model", "d_inner", "d_state", "d_conv", "dt_rank", "E", "K", "dtype",
-                 "gate_mode", "disc_mode", "flags", "reserved")]
+                 "gate_mode", "disc_mode", "flags", "small_proj_experts")]
 
 
 class RomWeights(ctypes.Structure):
@@ -81,15 +81,16 @@ def status_string(code: int) -> str:
     return lib().rom_status_string(int(code)).decode()
 
 
-def make_config(B, L, d_model, d_inner, d_state, d_conv, dt_rank, E, K, dtype, gate_mode=0, disc_mode=0, flags=0) -> RomConfig:
+def make_config(B, L, d_model, d_inner, d_state, d_conv, dt_rank, E, K, dtype, gate_mode=0, disc_mode=0, flags=0,
+                small_proj_experts=0) -> RomConfig:
     dt = {"f32": ROM_F32, "bf16": ROM_BF16, torch.float32: ROM_F32, torch.bfloat16: ROM_BF16}[dtype]
-    return RomConfig(B, L, d_model, d_inner, d_state, d_conv, dt_rank, E, K, dt, gate_mode, disc_mode, flags, 0)
+    return RomConfig(B, L, d_model, d_inner, d_state, d_conv, dt_rank, E, K, dt, gate_mode, disc_mode, flags, small_proj_experts)
 
 
-def config_from_shape(shape, gate_mode=0, disc_mode=0, flags=0) -> RomConfig:
-    """shape: a synth.RomShape."""
+def config_from_shape(shape, gate_mode=0, disc_mode=0, flags=0, small_proj_experts=0) -> RomConfig:
+    """shape: a synth.RomShape.  small_proj_experts: 0 = shared x Proj / dt Proj, shape.E = one per expert."""
     return make_config(shape.B, shape.L, shape.d_model, shape.d_inner, shape.d_state, shape.d_conv, shape.dt_rank,
-                       shape.E, shape.K, shape.dtype, gate_mode, disc_mode, flags)
+                       shape.E, shape.K, shape.dtype, gate_mode, disc_mode, flags, small_proj_experts)
 
 
 def _ptr(t: Optional[torch.Tensor], cuda: bool = True) -> Optional[int]:

@@ -45,6 +45,12 @@ WsLayout make_layout(const rom_config& c) {
   l.Ygp = take(l.esz * (size_t)l.rows_max * c.d_inner);
   l.Op = take(l.esz * (size_t)l.rows_max * c.d_model);
   l.scan_ws = take(sizeof(float) * scan_ws_floats(c.B, c.d_inner, c.L));
+  // per-expert x Proj / dt Proj: their outputs in expert order, summed over the K slots afterwards
+  const bool routed_small = c.small_proj_experts > 1;
+  l.delta_rp = take(routed_small ? l.esz * (size_t)l.rows_max * R : 0);
+  l.Bp = take(routed_small ? sizeof(float) * (size_t)l.rows_max * N : 0);
+  l.Cp = take(routed_small ? sizeof(float) * (size_t)l.rows_max * N : 0);
+  l.Dpre = take(routed_small ? sizeof(float) * (size_t)l.rows_max * c.d_inner : 0);
   l.total = o;
   return l;
 }
@@ -58,13 +64,16 @@ int check_config(const rom_config* c, int which) {
   if (!c) return ROM_ERR_INVALID_ARG;
   if (c->dtype != ROM_F32 && c->dtype != ROM_BF16) return ROM_ERR_INVALID_ARG;
   if (c->B < 1 || c->L < 1) return ROM_ERR_INVALID_ARG;
-  if (c->reserved != 0 || (c->flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
+  if ((c->flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
   if (which != 2) {
     if (c->E < 1 || c->K < 1 || c->K > c->E) return ROM_ERR_INVALID_ARG;
     if (c->E > kMaxE || c->K > kMaxK) return ROM_ERR_UNSUPPORTED;
     if (c->gate_mode != 0 && c->gate_mode != 1) return ROM_ERR_INVALID_ARG;
     if (c->d_model < 64 || c->d_model % 64 != 0) return ROM_ERR_INVALID_ARG;
     if ((int64_t)c->B * c->L * c->K >= (int64_t)1 << 30) return ROM_ERR_UNSUPPORTED;
+    if (c->small_proj_experts != 0 && c->small_proj_experts != 1 && c->small_proj_experts != c->E) return ROM_ERR_INVALID_ARG;
+  } else if (c->small_proj_experts < 0) {
+    return ROM_ERR_INVALID_ARG;
   }
   if (which != 1) {
     if (c->d_inner < 64 || c->d_inner % 64 != 0) return ROM_ERR_INVALID_ARG;
@@ -255,14 +264,29 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   // S4: un-permute + sum over selected experts + conv + SiLU
   ROM_CUDA(launch_conv(c, W + lay.XZp, in_token_order ? nullptr : row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
   ROM_STAGE_DONE();
-  // S5: x Proj -> delta_r | B | C
-  Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N, nullptr, nullptr};
-  ROM_CUDA(gemm(W + lay.U, De, w->W_x, De, 1, 0, T, R + 2 * N, De, nullptr, nullptr, e_x));
-  ROM_STAGE_DONE();
-  // S6: dt Proj + softplus
-  Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0, nullptr, nullptr};
-  ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
-  ROM_STAGE_DONE();
+  if (c.small_proj_experts <= 1) {
+    // S5: x Proj -> delta_r | B | C  (shared by all experts)
+    Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N, nullptr, nullptr};
+    ROM_CUDA(gemm(W + lay.U, De, w->W_x, De, 1, 0, T, R + 2 * N, De, nullptr, nullptr, e_x));
+    ROM_STAGE_DONE();
+    // S6: dt Proj + softplus
+    Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0, nullptr, nullptr};
+    ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
+    ROM_STAGE_DONE();
+  } else {
+    // Per-expert x Proj / dt Proj under the same routing: U rows gathered into expert order (in the buffer the
+    // scan fills later), two more grouped GEMMs over the existing row tiles, then the sum over the K slots.
+    ROM_CUDA(launch_gather_rows_to(c, W + lay.U, W + lay.Ygp, De, W, lay, st));
+    Epilogue e_x{EPI_XPROJ, W + lay.delta_rp, R, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp), nullptr, R, N, nullptr, nullptr};
+    ROM_CUDA(gemm(W + lay.Ygp, De, w->W_x, De, c.E, (int64_t)(R + 2 * N) * De, (int)lay.rows_max, R + 2 * N, De, tile_expert, num_m_tiles, e_x));
+    ROM_STAGE_DONE();
+    Epilogue e_dt{EPI_F32, W + lay.Dpre, De, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
+    ROM_CUDA(gemm(W + lay.delta_rp, R, w->W_dt, R, c.E, (int64_t)De * R, (int)lay.rows_max, De, R, tile_expert, num_m_tiles, e_dt));
+    ROM_CUDA(launch_small_combine(c, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp),
+                                  reinterpret_cast<float*>(W + lay.Dpre), row_of_assign, w->b_dt, reinterpret_cast<float*>(W + lay.Bm),
+                                  reinterpret_cast<float*>(W + lay.Cm), reinterpret_cast<float*>(W + lay.Delta), st));
+    ROM_STAGE_DONE();
+  }
   // S7 + S8 + S9: scan, gate, re-permute
   // K = 1: the gate row of a token is its Gate Proj row in expert order; K > 1: the summed rows from S4
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;

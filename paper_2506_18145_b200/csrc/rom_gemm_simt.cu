@@ -22,6 +22,9 @@ __device__ __forceinline__ void epi_store_scalar(const Epilogue& ep, int m, int 
       else if (n < ep.R + ep.N) ep.Bm[(size_t)m * ep.N + (n - ep.R)] = v;
       else ep.Cm[(size_t)m * ep.N + (n - ep.R - ep.N)] = v;
       break;
+    case EPI_F32:
+      reinterpret_cast<float*>(ep.C)[(size_t)m * ep.ldc + n] = v;
+      break;
     default:
       reinterpret_cast<float*>(ep.C)[(size_t)m * ep.ldc + n] = softplus_f(v + (ep.bias ? ep.bias[n] : 0.0f));
       break;

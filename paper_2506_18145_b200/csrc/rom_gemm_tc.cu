@@ -42,8 +42,9 @@ constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 // Operand stages and epilogue staging per output op.  The softplus epilogue (dt Proj: only two K blocks per tile,
 // and the one GEMM here whose time is its fp32 output) gives up one operand stage for a 32 x 32 fp32 staging
 // square per epilogue warp, through which its stores become whole 128-byte row segments.
-__host__ __device__ constexpr int stages_of(int mode) { return mode == EPI_SOFTPLUS ? 3 : MAX_STAGES; }
-__host__ __device__ constexpr int out_stage_bytes_of(int mode) { return mode == EPI_SOFTPLUS ? NUM_EPI_WARPS_C * 32 * 32 * 4 : 0; }
+__host__ __device__ constexpr bool f32_out(int mode) { return mode == EPI_SOFTPLUS || mode == EPI_F32; }
+__host__ __device__ constexpr int stages_of(int mode) { return f32_out(mode) ? 3 : MAX_STAGES; }
+__host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(mode) ? NUM_EPI_WARPS_C * 32 * 32 * 4 : 0; }
 __host__ __device__ constexpr int smem_bytes_of(int mode) {
   return stages_of(mode) * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
 }
@@ -187,13 +188,19 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
 // Softplus output op on a 32 (rows of this warp) x 32 (columns) accumulator square: every lane activates its row,
 // the square goes through a swizzled shared-memory staging area, and is written as whole 128-byte row segments
 // (8 lanes per row, 4 rows per store instruction) instead of 32 scattered 16-byte pieces.
+template <int MODE>
 __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, int row0, int M_valid, int n0, int N,
                                                const uint32_t (&r)[32], const float4 (&bq)[8], int lane) {
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
-    const float4 b = bq[c];
-    const float4 o = make_float4(softplus_fast(__uint_as_float(r[4 * c]) + b.x), softplus_fast(__uint_as_float(r[4 * c + 1]) + b.y),
-                                 softplus_fast(__uint_as_float(r[4 * c + 2]) + b.z), softplus_fast(__uint_as_float(r[4 * c + 3]) + b.w));
+    float4 o;
+    if constexpr (MODE == EPI_F32) {      // plain fp32 rows, no bias, no activation
+      o = make_float4(__uint_as_float(r[4 * c]), __uint_as_float(r[4 * c + 1]), __uint_as_float(r[4 * c + 2]), __uint_as_float(r[4 * c + 3]));
+    } else {
+      const float4 b = bq[c];
+      o = make_float4(softplus_fast(__uint_as_float(r[4 * c]) + b.x), softplus_fast(__uint_as_float(r[4 * c + 1]) + b.y),
+                      softplus_fast(__uint_as_float(r[4 * c + 2]) + b.z), softplus_fast(__uint_as_float(r[4 * c + 3]) + b.w));
+    }
     *reinterpret_cast<float4*>(sw + lane * 32 + ((c ^ (lane & 7)) << 2)) = o;
   }
   __syncwarp();
@@ -355,14 +362,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);     // in flight together with the tensor-memory load
         tmem_ld_wait(ra);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
-        if (MODE == EPI_SOFTPLUS) epi_softplus32(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
+        if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
         else if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale, bq);
         ch += 2;
         if (ch >= n_chunks) break;
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);
         tmem_ld_wait(rb);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
-        if (MODE == EPI_SOFTPLUS) epi_softplus32(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
+        if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
         else if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale, bq);
         ch += 2;
       }
@@ -436,7 +443,7 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   }
   auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
               : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : epi.mode == EPI_OUTPROJ ? gemm_tc_kernel<EPI_OUTPROJ>
-              : gemm_tc_kernel<EPI_SOFTPLUS>;
+              : epi.mode == EPI_F32 ? gemm_tc_kernel<EPI_F32> : gemm_tc_kernel<EPI_SOFTPLUS>;
   const int smem_bytes = smem_bytes_of(epi.mode);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;

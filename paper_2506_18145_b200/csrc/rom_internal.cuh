@@ -50,6 +50,7 @@ struct WsLayout {
   size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts, chunk_prob, wr_f64;
   size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
   size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op, scan_ws;
+  size_t delta_rp, Bp, Cp, Dpre;      // per-expert x Proj / dt Proj only
   size_t total;
   int64_t T, A, rows_max, max_m_tiles, n_chunks;
   size_t esz;
@@ -66,8 +67,9 @@ enum EpiMode : int {
   EPI_SOFTPLUS = 2,   // Delta[m, n] = softplus(acc + bias[n])  (fp32)
   EPI_INPROJ = 3,     // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype); with row_token
                       // (tensor path, top-1) row m is written at row row_token[m], i.e. back in token order
-  EPI_OUTPROJ = 4     // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
+  EPI_OUTPROJ = 4,    // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
                       // row_token[m] < 0 (segment padding) are skipped   (dtype; tensor path only)
+  EPI_F32 = 5         // C[m, n] = acc                          (fp32)
 };
 struct Epilogue {
   int mode;
@@ -95,6 +97,14 @@ cudaError_t launch_balance(const rom_config& c, const void* x, const void* W_r, 
                            float* F, float* Pbar, float* loss, char* ws, const WsLayout& lay, cudaStream_t st);
 
 cudaError_t launch_gather_rows(const rom_config& c, const void* x, char* ws, const WsLayout& lay, cudaStream_t st);
+// dst[row, :] = src[token of row, :] for rows of `width` dtype elements (zero rows in the padding); dst has rows_max rows.
+cudaError_t launch_gather_rows_to(const rom_config& c, const void* src, void* dst, int width, char* ws, const WsLayout& lay,
+                                  cudaStream_t st);
+// Per-expert x Proj / dt Proj: sums over the K slots of a token, in ascending slot order (fp32):
+//   Bm[t, :] = sum_k Bp[row(t,k), :],  Cm likewise,  Delta[t, c] = softplus(b_dt[c] + sum_k Dpre[row(t,k), c]).
+cudaError_t launch_small_combine(const rom_config& c, const float* Bp, const float* Cp, const float* Dpre,
+                                 const int32_t* row_of_assign, const float* b_dt, float* Bm, float* Cm, float* Delta,
+                                 cudaStream_t st);
 
 // C[M,N] = A[M,Kd] * B[e][N,Kd]^T, A and B K-contiguous.  Grouped when tile_expert != nullptr: row tile
 // i (kTileM rows) uses expert tile_expert[i]; the number of valid row tiles is *num_m_tiles_dev.

@@ -402,10 +402,15 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
 }
 
 cudaError_t launch_gather_rows(const rom_config& c, const void* x, char* ws, const WsLayout& lay, cudaStream_t st) {
-  const int vec_per_row = (int)((size_t)c.d_model * lay.esz / 16);
+  return launch_gather_rows_to(c, x, ws + lay.x_perm, c.d_model, ws, lay, st);
+}
+
+cudaError_t launch_gather_rows_to(const rom_config& c, const void* src, void* dst, int width, char* ws, const WsLayout& lay,
+                                  cudaStream_t st) {
+  const int vec_per_row = (int)((size_t)width * lay.esz / 16);
   const int wpb = 8;
   const int blocks = (int)((lay.rows_max + wpb - 1) / wpb);
-  gather_rows<<<blocks, wpb * 32, 0, st>>>(reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(ws + lay.x_perm),
+  gather_rows<<<blocks, wpb * 32, 0, st>>>(reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst),
                                           reinterpret_cast<const int32_t*>(ws + lay.assign_of_row),
                                           reinterpret_cast<const int32_t*>(ws + lay.pad_offsets), c.E, c.K, vec_per_row,
                                           (int)lay.rows_max);

@@ -82,7 +82,8 @@ extern "C" int rom_route_noalloc(const rom_config* cfg, const void* x, const voi
   if (c.B < 1 || c.L < 1 || c.E < 1 || c.K < 1 || c.K > c.E) return ROM_ERR_INVALID_ARG;
   if (c.gate_mode != 0 && c.gate_mode != 1) return ROM_ERR_INVALID_ARG;
   if (c.d_model < 64 || c.d_model % 64 != 0) return ROM_ERR_INVALID_ARG;
-  if (c.reserved != 0 || (c.flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
+  if ((c.flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
+  if (c.small_proj_experts != 0 && c.small_proj_experts != 1 && c.small_proj_experts != c.E) return ROM_ERR_INVALID_ARG;
   if (c.E > kMaxE || c.K > kMaxK) return ROM_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(x) & 15u) || (reinterpret_cast<uintptr_t>(W_r) & 15u)) return ROM_ERR_INVALID_ARG;
   // the built-in scratch has a fixed size: larger problems must use rom_route with a caller workspace

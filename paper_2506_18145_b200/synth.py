@@ -80,7 +80,8 @@ def _rand(seed: int, size) -> torch.Tensor:
     return torch.rand(size, generator=g, dtype=torch.float32)
 
 
-def make_inputs(shape: RomShape, recipe: str = "paper", with_D: bool = True) -> Dict[str, Optional[torch.Tensor]]:
+def make_inputs(shape: RomShape, recipe: str = "paper", with_D: bool = True,
+                routed_small: bool = False) -> Dict[str, Optional[torch.Tensor]]:
     """Draw x and every weight of one RoM layer on the CPU.
 
     recipe "paper": x ~ N(0,1); all projection / conv / router weights ~ N(0, 0.02^2);
@@ -96,6 +97,8 @@ def make_inputs(shape: RomShape, recipe: str = "paper", with_D: bool = True) -> 
         x[B,L,D_m]  W_r[E,D_m]  W_inz[E,2*D_e,D_m] (rows [0,D_e) Conv Proj, [D_e,2D_e) Gate Proj)
         w_conv[k,D_e] (tap k-1 multiplies the current token)  W_x[R+2N, D_e] (rows delta|B|C)
         W_dt[D_e,R]  W_out[E,D_m,D_e]  A[D_e,N]  D[D_e]  b_conv[D_e]  b_dt[D_e]  b_r[E] or None
+    routed_small: W_x[E, R+2N, D_e] and W_dt[E, D_e, R], one x Proj / dt Proj per expert (the
+        ablation row of Section 5.3), same distributions.
     """
     s = shape
     dt = torch_dtype(s)
@@ -115,8 +118,9 @@ def make_inputs(shape: RomShape, recipe: str = "paper", with_D: bool = True) -> 
     out["W_r"] = _randn(sb + _TID["W_r"], (s.E, s.d_model), std["W_r"]).to(dt)
     out["W_inz"] = _randn(sb + _TID["W_inz"], (s.E, 2 * s.d_inner, s.d_model), std["W_inz"]).to(dt)
     out["w_conv"] = _randn(sb + _TID["w_conv"], (s.d_conv, s.d_inner), std["w_conv"]).to(dt)
-    out["W_x"] = _randn(sb + _TID["W_x"], (R + 2 * N, s.d_inner), std["W_x"]).to(dt)
-    out["W_dt"] = _randn(sb + _TID["W_dt"], (s.d_inner, R), std["W_dt"]).to(dt)
+    lead = (s.E,) if routed_small else ()
+    out["W_x"] = _randn(sb + _TID["W_x"], lead + (R + 2 * N, s.d_inner), std["W_x"]).to(dt)
+    out["W_dt"] = _randn(sb + _TID["W_dt"], lead + (s.d_inner, R), std["W_dt"]).to(dt)
     out["W_out"] = _randn(sb + _TID["W_out"], (s.E, s.d_model, s.d_inner), std["W_out"]).to(dt)
 
     out["A"] = -(torch.arange(1, N + 1, dtype=torch.float32)).repeat(s.d_inner, 1).contiguous()

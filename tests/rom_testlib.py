@@ -46,7 +46,8 @@ class GpuLayer:
 
     def __init__(self, shape, p, gate_mode=0, disc_mode=0, flags=0, device="cuda"):
         self.shape = shape
-        self.cfg = rb.config_from_shape(shape, gate_mode, disc_mode, flags)
+        # three-dimensional W_x: one x Proj / dt Proj per expert
+        self.cfg = rb.config_from_shape(shape, gate_mode, disc_mode, flags, shape.E if p["W_x"].dim() == 3 else 0)
         self.dev = {k: (None if v is None else v.to(device).contiguous()) for k, v in p.items()}
         self.weights = rb.make_weights(self.dev)
         self.ws = rb.alloc_workspace(self.cfg, device)

@@ -151,8 +151,8 @@ def test_scan_long_memory_small_delta():
 
 
 # ---------------------------------------------------------------------------------------------- layer
-def check_layer(s, recipe, with_D=True, gate_mode=0, disc_mode=0, flags=0, check_taps=True):
-    p = synth.make_inputs(s, recipe=recipe, with_D=with_D)
+def check_layer(s, recipe, with_D=True, gate_mode=0, disc_mode=0, flags=0, check_taps=True, routed_small=False):
+    p = synth.make_inputs(s, recipe=recipe, with_D=with_D, routed_small=routed_small)
     ref, im = oracle_layer(s, p, gate_mode, disc_mode)
     g = GpuLayer(s, p, gate_mode, disc_mode, flags)
     out = g.forward()
@@ -196,6 +196,35 @@ def test_layer_small_shapes(kw, dtype, flags):
 def test_layer_modes(gate_mode, disc_mode, dtype):
     s = small_shape(dtype=dtype, L=200)
     check_layer(s, "unit", gate_mode=gate_mode, disc_mode=disc_mode)
+
+
+# per-expert x Proj / dt Proj (the "(Conv, Gate, dt, x, Out)" ablation row of Section 5.3)
+@pytest.mark.parametrize("kw", [
+    dict(),                                                       # K = 2, ragged L
+    dict(E=8, K=1, B=3, L=130),
+    dict(E=3, K=3, L=64, d_conv=3),
+    dict(E=4, K=1, dt_rank=32, B=1, L=1),                         # one token
+    dict(E=6, K=2, router_bias_scale=4.0, L=513),                 # skewed loads, some experts nearly empty
+])
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
+def test_layer_routed_small_projections(kw, dtype, flags):
+    s = small_shape(dtype=dtype, **kw)
+    check_layer(s, "unit", flags=flags, routed_small=True)
+
+
+def test_layer_routed_small_projections_small_bf16_config():
+    check_layer(synth.CONFIGS["small_bf16"], "unit", routed_small=True)
+
+
+def test_layer_routed_small_with_identical_experts_matches_shared_path_on_gpu():
+    """E copies of one x Proj / dt Proj, top-1: the per-expert path must reproduce the shared path's rows."""
+    s = small_shape(E=4, K=1, L=400)
+    p = synth.make_inputs(s, recipe="unit")
+    shared = GpuLayer(s, p).forward().clone()
+    q = dict(p)
+    q["W_x"] = p["W_x"][None].repeat(s.E, 1, 1).contiguous(); q["W_dt"] = p["W_dt"][None].repeat(s.E, 1, 1).contiguous()
+    routed = GpuLayer(s, q).forward()
+    assert_close(np64(routed), np64(shared), 1e-2, "per-expert vs shared")
 
 
 def test_layer_single_expert_is_dense_mamba_on_gpu():
