@@ -39,7 +39,6 @@ inline int scan_chunks(int B, int De, int L) {
   }
   return best;
 }
-inline int scan_chunk_len(int L, int nch) { return (int)align_up((size_t)(L + nch - 1) / nch, 64); }
 inline size_t scan_ws_floats(int B, int De, int L) {
   const int nch = scan_chunks(B, De, L);
   return nch == 1 ? 0 : (size_t)B * nch * De * (2 * 16 + 1);

@@ -29,6 +29,8 @@
 // both bank-conflict free.
 #include <type_traits>
 
+#include <cmath>
+
 #include "rom_internal.cuh"
 
 namespace rom {
@@ -115,6 +117,7 @@ struct ScanArgs {
   const void* z; int ldz; const int32_t* z_row; const float* h0; void* y; float* h_last; const int32_t* y_rows;
   int K, L, De;
   int Lc, nch;          // chunk length and chunks per sequence (nch == 1: Lc == L); blockIdx.z = chunk
+  int L0;               // length of chunk 0; chunk j >= 1 covers steps [L0 + (j-1) Lc, L0 + j Lc)
   float* sum_delta;     // state-only blocks: [B*nch, De] sum of Delta over the chunk
   int gate_activated;   // z already holds SiLU(gate pre-activation): multiply only
   int chunk_off;        // chunk of blockIdx.z == 0
@@ -145,10 +148,11 @@ scan_kernel(const ScanArgs p) {
   const int chunk = blockIdx.z + p.chunk_off;
   const bool so = MODE == 1 || (MODE == 2 && chunk != 0);  // this block only produces its end state
   const T* __restrict__ z = so ? nullptr : static_cast<const T*>(p.z);
-  const int L = min(p.Lc, p.L - chunk * p.Lc);            // steps of this chunk
+  const int t_first = chunk == 0 ? 0 : p.L0 + (chunk - 1) * p.Lc;
+  const int L = min(chunk == 0 ? p.L0 : p.Lc, p.L - t_first);   // steps of this chunk (<= 0: an empty chunk)
   const int b = blockIdx.y * p.nch + chunk;               // index of the (sequence, chunk) state
   const int c_base = blockIdx.x * CH;
-  const size_t tok0 = (size_t)blockIdx.y * p.L + (size_t)chunk * p.Lc;
+  const size_t tok0 = (size_t)blockIdx.y * p.L + (size_t)t_first;
 
   // ---- compute role: NC adjacent channels from block-local channel cl, states [g*NS, g*NS+NS)
   const int cl = (tid / S) * NC, g = tid % S;
@@ -428,6 +432,8 @@ cudaError_t launch_one(const ScanArgs& a, int B, int grid_z, cudaStream_t st) {
 
 // Work per thread, NC channels x NS states, as NC * 100 + NS: the largest of 1x8, 1x4, 1x2 that still
 // gives every SM sub-partition about two warps.
+constexpr double kFirstChunkRatio = 0.7;
+
 int pick_thread_shape(int B, int De, int num_sms) {
   const long long want_warps = 2LL * 4 * num_sms;
   const int shapes[2][2] = {{1, 8}, {1, 4}};
@@ -456,7 +462,7 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
   const bool zoh = c.disc_mode == 0;
   const int nch = chunk_ws ? scan_chunks(c.B, c.d_inner, c.L) : 1;
   if (nch == 1) {
-    a.Lc = c.L; a.nch = 1;
+    a.Lc = c.L; a.L0 = c.L; a.nch = 1;
     const int shape = pick_thread_shape(c.B, c.d_inner, num_sms);
     return zoh ? launch_shape<T, PRECISE, true>(shape, a, c.B, st) : launch_shape<T, PRECISE, false>(shape, a, c.B, st);
   }
@@ -466,7 +472,12 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
   float* h_end = chunk_ws;
   float* h_in = chunk_ws + n_state;
   float* sum_delta = chunk_ws + 2 * n_state;
-  a.Lc = scan_chunk_len(c.L, nch); a.nch = nch;
+  // Chunk 0 runs in full inside the first launch, next to state-only chunks that cost less per step: it is made
+  // shorter by kFirstChunkRatio so that its blocks do not outlast the others.
+  const double x = (double)c.L / ((double)(nch - 1) + kFirstChunkRatio);
+  a.Lc = (int)align_up((size_t)ceil(x), 64);
+  a.L0 = (int)align_up((size_t)ceil(kFirstChunkRatio * x), 64);
+  a.nch = nch;
   const int n_end = h_last ? nch : nch - 1;       // the last chunk's end state is only needed for h_last
   ScanArgs pa = a;
   pa.h_last = h_end; pa.sum_delta = sum_delta; pa.chunk_off = 0;
@@ -494,7 +505,7 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, 
     e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
   }
-  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, nullptr, gate_activated ? 1 : 0, 0};
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0};
   return c.dtype == ROM_BF16 ? launch_scan_t<__nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
                              : launch_scan_t<float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
 }
