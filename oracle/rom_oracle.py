@@ -32,7 +32,9 @@ identical experts, geometric-series closed form, exact ODE solution for ZOH,
 identity conv tap + causality, permutation tables vs brute force and a stable
 sort, gate sums, tie rule, two-half scan, parameter counts printed in the paper;
 per-expert small projections: E=1 / identical experts reduce to the shared form, rows of
-one expert equal the shared form with that expert's matrices, per-token brute force.
+one expert equal the shared form with that expert's matrices, per-token brute force;
+FFN-MoE with shared routing: library SwiGLU for E=1, per-token loops, identical experts with
+gates summing to one = the dense FFN, linearity in the gates.
 """
 from __future__ import annotations
 
@@ -341,6 +343,37 @@ def rom_layer_forward(x, W_r, b_r, W_inz, w_conv, b_conv, W_x, W_dt, b_dt, A, D,
     return out, dict(idx=idx, gate=gate, P=P, logit=logit, counts=counts, offsets=offsets,
                      perm=perm, inv_perm=inv, H=H, Zpre=Zpre, U=U.reshape(T, De), delta=delta,
                      Bm=Bm, Cm=Cm, Delta=Delta, Y=Y.reshape(T, De), Yg=Yg, h_last=h_last)
+
+
+# --------------------------------------------------------------------------- FFN-MoE with shared routing
+def ffn_moe_shared_routing(x, W_gu, W_down, idx, gate):
+    """Feed-forward SwiGLU mixture of experts that reuses the routing decision of the preceding RoM
+    layer (Appendix A.2, the two equations of the hybrid "RoM + FFN-MoE" model):
+        Y_t = sum_i R_i * E_i(X_t),   E_i(X_t) = 1[i in TopK] * f_i(X_t),
+    with idx[T,K] (the selected experts) and gate[T,K] (R_i of the selected experts) taken from that
+    layer's router, not recomputed.  The paper names f_i "the i-th feedforward SwiGLU expert" without
+    writing it out; the usual bias-free form is taken:
+        f_i(x) = W_down,i ( SiLU(W_gate,i x) * (W_up,i x) ).
+    x[T,D_m]; W_gu[E, 2*D_ff, D_m], rows [0,D_ff) = W_gate,i and [D_ff,2D_ff) = W_up,i;
+    W_down[E, D_m, D_ff].  Returns Y[T,D_m].
+    """
+    x = np.asarray(x, dtype=F64)
+    W_gu = np.asarray(W_gu, dtype=F64)
+    W_down = np.asarray(W_down, dtype=F64)
+    gate = np.asarray(gate, dtype=F64)
+    T, Dm = x.shape
+    E, twoF, _ = W_gu.shape
+    Dff = twoF // 2
+    Y = np.zeros((T, Dm), dtype=F64)
+    for k in range(idx.shape[1]):
+        for e in range(E):
+            tok = np.nonzero(idx[:, k] == e)[0]
+            if tok.size == 0:
+                continue
+            gu = x[tok] @ W_gu[e].T
+            hidden = silu(gu[:, :Dff]) * gu[:, Dff:]
+            Y[tok] += gate[tok, k][:, None] * (hidden @ W_down[e].T)
+    return Y
 
 
 # --------------------------------------------------------------------------- wiring pin

@@ -428,6 +428,59 @@ def test_layer_with_identical_small_experts_equals_shared_layer():
     np.testing.assert_allclose(run_layer(q1, K=1, R=s1["R"]), ref, rtol=1e-10, atol=1e-12)
 
 
+# ---------------------------------------------------------------------------------------------- FFN-MoE, shared routing
+def _ffn_case(seed, T=19, Dm=6, Dff=10, E=4, K=2):
+    g = rng(seed)
+    x = g.normal(size=(T, Dm)); W_gu = g.normal(size=(E, 2 * Dff, Dm)); W_down = g.normal(size=(E, Dm, Dff))
+    idx = np.stack([g.permutation(E)[:K] for _ in range(T)]).astype(np.int32)
+    gate = g.uniform(0.1, 1.0, size=(T, K))
+    return x, W_gu, W_down, idx, gate
+
+
+def test_ffn_moe_single_expert_is_library_swiglu():
+    x, W_gu, W_down, _, _ = _ffn_case(31, E=1, K=1)
+    T, Dff = x.shape[0], W_down.shape[2]
+    idx = np.zeros((T, 1), dtype=np.int32); gate = np.ones((T, 1))
+    Y = O.ffn_moe_shared_routing(x, W_gu, W_down, idx, gate)
+    xt = torch.tensor(x)
+    ref = (F.silu(xt @ torch.tensor(W_gu[0, :Dff]).T) * (xt @ torch.tensor(W_gu[0, Dff:]).T)) @ torch.tensor(W_down[0]).T
+    np.testing.assert_allclose(Y, ref.numpy(), rtol=1e-12, atol=1e-13)
+
+
+def test_ffn_moe_vs_per_token_loops():
+    x, W_gu, W_down, idx, gate = _ffn_case(32)
+    T, Dm = x.shape; Dff = W_down.shape[2]; K = idx.shape[1]
+    Y = O.ffn_moe_shared_routing(x, W_gu, W_down, idx, gate)
+    for t in range(T):
+        y = np.zeros(Dm)
+        for k in range(K):
+            e = idx[t, k]
+            hid = np.zeros(Dff)
+            for j in range(Dff):
+                a = float(W_gu[e, j] @ x[t]); b = float(W_gu[e, Dff + j] @ x[t])
+                hid[j] = a / (1.0 + math.exp(-a)) * b
+            y += gate[t, k] * (W_down[e] @ hid)
+        np.testing.assert_allclose(Y[t], y, rtol=1e-12, atol=1e-13)
+
+
+def test_ffn_moe_identical_experts_and_gate_linearity():
+    x, W_gu, W_down, idx, gate = _ffn_case(33)
+    W_gu[:] = W_gu[0]; W_down[:] = W_down[0]
+    gate = gate / gate.sum(axis=1, keepdims=True)          # gates summing to one: the mixture is the dense FFN
+    Y = O.ffn_moe_shared_routing(x, W_gu, W_down, idx, gate)
+    T = x.shape[0]
+    dense = O.ffn_moe_shared_routing(x, W_gu[:1], W_down[:1], np.zeros((T, 1), dtype=np.int32), np.ones((T, 1)))
+    np.testing.assert_allclose(Y, dense, rtol=1e-12, atol=1e-13)
+    # the output is linear in the gates and vanishes with them; the experts themselves are not gate-weighted inside
+    x2, W_gu2, W_down2, idx2, gate2 = _ffn_case(34)
+    Y2 = O.ffn_moe_shared_routing(x2, W_gu2, W_down2, idx2, gate2)
+    np.testing.assert_allclose(O.ffn_moe_shared_routing(x2, W_gu2, W_down2, idx2, 3.0 * gate2), 3.0 * Y2, rtol=1e-12)
+    assert np.abs(O.ffn_moe_shared_routing(x2, W_gu2, W_down2, idx2, 0.0 * gate2)).max() == 0.0
+    # swapping the two halves of W_gu (gate <-> up) changes the result: SiLU sits on the first half
+    W_sw = np.concatenate([W_gu2[:, W_down2.shape[2]:], W_gu2[:, :W_down2.shape[2]]], axis=1)
+    assert np.abs(O.ffn_moe_shared_routing(x2, W_sw, W_down2, idx2, gate2) - Y2).max() > 1e-3
+
+
 # ---------------------------------------------------------------------------------------------- P11
 def test_wiring_reproduces_paper_parameter_counts():
     rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_param_counts.txt")) if l.strip() and not l.startswith("#")]
