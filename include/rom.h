@@ -166,6 +166,25 @@ ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const
                       int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
                       void *ws, size_t ws_bytes, void *stream);
 
+/* Feed-forward SwiGLU mixture of experts that shares the routing decision of the preceding RoM layer
+ * (Appendix A.2, the two equations of the hybrid RoM + FFN-MoE model):
+ *   Y_t = sum_i R_i * 1[i in TopK] * f_i(X_t),   f_i(x) = W_down,i ( SiLU(W_gate,i x) * (W_up,i x) )
+ * (the paper names f_i a SwiGLU expert without writing it out; the usual bias-free form is taken).
+ * The selected experts and their gates are not recomputed: topk_idx [T,K] i32 and gates [T,K] f32 are
+ * the outputs of that layer's rom_route / rom_layer_forward call (device pointers, read only).
+ *   d_ff   : hidden width of an expert, a multiple of 128
+ *   W_gu   : [E, 2*d_ff, d_model] dtype, rows [0,d_ff) = W_gate,i, rows [d_ff,2*d_ff) = W_up,i
+ *   W_down : [E, d_model, d_ff]   dtype
+ *   x, out : [B, L, d_model]      dtype (x is this layer's own input)
+ *   ws     : rom_ffn_moe_workspace_size(cfg, d_ff) bytes of scratch, independent of the RoM layer's
+ * Uses cfg->B, L, d_model, E, K, dtype, flags.  The K experts of a token must be distinct and in
+ * [0, E); an index outside that range is clamped (every access stays in bounds, the result for that
+ * token is unspecified) and rom_get_status then reports ROM_ERR_INVALID_ARG.                        */
+ROM_API int rom_ffn_moe_workspace_size(const rom_config *cfg, int32_t d_ff, size_t *bytes);
+ROM_API int rom_ffn_moe_forward(const rom_config *cfg, int32_t d_ff, const void *W_gu, const void *W_down,
+                        const void *x, const int32_t *topk_idx, const float *gates, void *out,
+                        void *ws, size_t ws_bytes, void *stream);
+
 /* Profiling aid: the same launch sequence as rom_layer_forward with a CUDA event recorded on
  * `stream` between stages; synchronises the stream and writes the device time of each stage in
  * milliseconds to stage_ms (host out, at least rom_num_stages() floats).  Stage i is named

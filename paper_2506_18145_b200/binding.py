@@ -21,7 +21,8 @@ ROM_OK = 0
 
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
-           "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance")
+           "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance",
+           "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward")
 
 
 class RomConfig(ctypes.Structure):
@@ -58,6 +59,8 @@ def lib() -> ctypes.CDLL:
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
         L.rom_route_noalloc.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
         L.rom_route_balance.argtypes = [cfgp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, ctypes.c_size_t, vp]
+        L.rom_ffn_moe_workspace_size.argtypes = [cfgp, ctypes.c_int32, szp]
+        L.rom_ffn_moe_forward.argtypes = [cfgp, ctypes.c_int32, vp, vp, vp, i32p, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_scan.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_layer_forward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, i32p, vp, i32p, vp, ctypes.c_size_t, vp]
         L.rom_workspace_find.argtypes = [cfgp, ctypes.c_char_p, szp, szp]
@@ -170,6 +173,22 @@ def rom_layer_forward(cfg, weights: RomWeights, x, out, topk_idx_out, gates_out,
                                  _ptr(gates_out), _ptr(counts_out), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_layer_forward")
+    return rc
+
+
+def ffn_moe_workspace_size(cfg: RomConfig, d_ff: int) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().rom_ffn_moe_workspace_size(ctypes.byref(cfg), int(d_ff), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_ffn_moe_workspace_size")
+    return int(n.value)
+
+
+def rom_ffn_moe_forward(cfg, d_ff, W_gu, W_down, x, topk_idx, gates, out, ws, stream=None, check=True) -> int:
+    rc = lib().rom_ffn_moe_forward(ctypes.byref(cfg), int(d_ff), _ptr(W_gu), _ptr(W_down), _ptr(x), _ptr(topk_idx), _ptr(gates),
+                                   _ptr(out), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_ffn_moe_forward")
     return rc
 
 

@@ -352,7 +352,7 @@ int rom_get_status(void* ws, void* stream, int32_t* host_code) {
   ROM_CUDA(cudaMemcpyAsync(v, ws, sizeof(v), cudaMemcpyDeviceToHost, st));
   ROM_CUDA(cudaStreamSynchronize(st));
   ROM_CUDA(cudaMemsetAsync(ws, 0, sizeof(int32_t) * kStatusInts, st));
-  *host_code = v[kStatCode] == 0 ? ROM_OK : ROM_ERR_DEVICE_TIMEOUT;
+  *host_code = v[kStatCode];      // 0, or the rom_status a kernel latched
   return ROM_OK;
 }
 

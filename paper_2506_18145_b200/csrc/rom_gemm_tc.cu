@@ -240,7 +240,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   int num_m_tiles = (M_max + BLOCK_M - 1) / BLOCK_M;
   if (num_m_tiles_dev) num_m_tiles = min(num_m_tiles, *num_m_tiles_dev);
   const int M_valid = min(M_max, num_m_tiles * BLOCK_M);
-  const int n_tiles = (N + block_n - 1) / block_n;
+  // EPI_SWIGLU: a tile holds 128 gate columns and the 128 up columns of the same hidden units
+  const int n_tiles = MODE == EPI_SWIGLU ? N / 128 : (N + block_n - 1) / block_n;
   const int total_tiles = num_m_tiles * n_tiles;
   const int num_kb = (Kd + BLOCK_K - 1) / BLOCK_K;
   const uint32_t stage_tx = A_STAGE_BYTES + (uint32_t)block_n * BLOCK_K * 2;
@@ -270,13 +271,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const int m_tile = tile / n_tiles, n_tile = tile % n_tiles;
         const int e = tile_expert ? tile_expert[m_tile] : 0;
-        const int b_row = e * N + n_tile * block_n;
+        const int b_row = MODE == EPI_SWIGLU ? e * 2 * N + n_tile * 128 : e * N + n_tile * block_n;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), stage_tx);
           const uint32_t sa = base + stage * STAGE_BYTES;
           tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BLOCK_K, m_tile * BLOCK_M);
           tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row);
+          if (MODE == EPI_SWIGLU)     // second half of the B tile: the up rows of the same 128 hidden units (box = 128 rows)
+            tma_load_2d(sa + A_STAGE_BYTES + 128 * BLOCK_K * 2, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row + N);
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -355,7 +358,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const int n_base = n_tile * block_n;
       uint32_t ra[32], rb[32];
       float4 bq[8];
-      int ch = half;
+      if constexpr (MODE == EPI_SWIGLU) {
+        // accumulator columns [0,128) = gate, [128,256) = up; this warp takes 32-column groups half and half + 2
+        for (int c = half; c < 4; c += 2) {
+          tmem_ld32_issue(taddr + c * 32, ra);
+          tmem_ld32_issue(taddr + 128 + c * 32, rb);
+          tmem_ld_wait(ra);
+          tmem_ld_wait(rb);
+          if (row_ok) {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(ep.C) + out_row * ep.ldc + n_tile * 128 + c * 32;
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              uint4 q;
+              uint32_t* w = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const float v0 = silu_fast(__uint_as_float(ra[j + 2 * i])) * __uint_as_float(rb[j + 2 * i]);
+                const float v1 = silu_fast(__uint_as_float(ra[j + 2 * i + 1])) * __uint_as_float(rb[j + 2 * i + 1]);
+                __nv_bfloat162 hh = __floats2bfloat162_rn(v0, v1);
+                w[i] = *reinterpret_cast<uint32_t*>(&hh);
+              }
+              *reinterpret_cast<uint4*>(dst + j) = q;
+            }
+          }
+        }
+      }
+      int ch = MODE == EPI_SWIGLU ? n_chunks : half;
       if (ch < n_chunks) tmem_ld32_issue(taddr + ch * 32, ra);
       // two register buffers: while one chunk is processed the next chunk's tensor-memory load is in flight
       while (ch < n_chunks) {
@@ -427,10 +455,13 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
                            const int32_t* tile_expert, const int32_t* num_m_tiles_dev, const Epilogue& epi,
                            int32_t* status, cudaStream_t st) {
   // N tile: a multiple of 32 (epilogue column groups) and of 16 (UMMA N for M = 128), at most 256
-  int block_n = N >= MAX_BLOCK_N ? MAX_BLOCK_N : (N + 31) / 32 * 32;
+  const bool swiglu = epi.mode == EPI_SWIGLU;      // N output columns from 2N rows of B per expert, loaded as two boxes of 128 rows
+  if (swiglu && (N % 128 != 0 || MAX_BLOCK_N != 256)) return cudaErrorInvalidValue;
+  int block_n = (swiglu || N >= MAX_BLOCK_N) ? MAX_BLOCK_N : (N + 31) / 32 * 32;
   CUtensorMap ta, tb;
   if (!make_tmap(&ta, A, (uint64_t)M_max, (uint64_t)Kd, (uint64_t)lda, BLOCK_M)) return cudaErrorInvalidValue;
-  if (!make_tmap(&tb, Bw, (uint64_t)n_experts * N, (uint64_t)Kd, (uint64_t)ldb, (uint32_t)block_n)) return cudaErrorInvalidValue;
+  if (!make_tmap(&tb, Bw, (uint64_t)n_experts * (swiglu ? 2 * N : N), (uint64_t)Kd, (uint64_t)ldb, swiglu ? 128u : (uint32_t)block_n))
+    return cudaErrorInvalidValue;
   // instruction descriptor: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
   static int num_sms = 0;
@@ -443,11 +474,12 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   }
   auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
               : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : epi.mode == EPI_OUTPROJ ? gemm_tc_kernel<EPI_OUTPROJ>
-              : epi.mode == EPI_F32 ? gemm_tc_kernel<EPI_F32> : gemm_tc_kernel<EPI_SOFTPLUS>;
+              : epi.mode == EPI_F32 ? gemm_tc_kernel<EPI_F32> : epi.mode == EPI_SWIGLU ? gemm_tc_kernel<EPI_SWIGLU>
+              : gemm_tc_kernel<EPI_SOFTPLUS>;
   const int smem_bytes = smem_bytes_of(epi.mode);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
-  const int n_tiles = (N + block_n - 1) / block_n;
+  const int n_tiles = swiglu ? N / 128 : (N + block_n - 1) / block_n;
   const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
   const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
   kern<<<grid, NUM_THREADS, smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);

@@ -16,7 +16,7 @@ constexpr int kMaxK = 8;
 constexpr int kStatusInts = 64;    // status block at the head of the workspace
 
 // status word slots
-constexpr int kStatCode = 0;       // 0 or ROM_ERR_DEVICE_TIMEOUT
+constexpr int kStatCode = 0;       // 0 or the rom_status a kernel latched (a wait that expired, an index out of range)
 constexpr int kStatWhere = 1;      // which wait gave up (debug aid)
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -68,7 +68,9 @@ enum EpiMode : int {
                       // (tensor path, top-1) row m is written at row row_token[m], i.e. back in token order
   EPI_OUTPROJ = 4,    // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
                       // row_token[m] < 0 (segment padding) are skipped   (dtype; tensor path only)
-  EPI_F32 = 5         // C[m, n] = acc                          (fp32)
+  EPI_F32 = 5,        // C[m, n] = acc                          (fp32)
+  EPI_SWIGLU = 6      // C[m, j] = SiLU(acc[m, j]) * acc[m, N + j], j < N: B holds, per expert, N "gate" rows then N "up"
+                      // rows; N % 128 == 0   (dtype; tensor path only)
 };
 struct Epilogue {
   int mode;
@@ -94,6 +96,11 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
 // Router + load-balance statistic: F[E], Pbar[E], loss[1] (device fp32, each may be null).
 cudaError_t launch_balance(const rom_config& c, const void* x, const void* W_r, const float* b_r, float alpha,
                            float* F, float* Pbar, float* loss, char* ws, const WsLayout& lay, cudaStream_t st);
+
+// Permutation tables from a routing decision made elsewhere: topk_idx [T, K] (device) -> the same tables launch_route
+// leaves in the workspace (counts, offsets, padded offsets, row tiles, row <-> assignment maps).
+cudaError_t launch_perm_from_idx(const rom_config& c, const int32_t* topk_idx, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                 int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st);
 
 cudaError_t launch_gather_rows(const rom_config& c, const void* x, char* ws, const WsLayout& lay, cudaStream_t st);
 // dst[row, :] = src[token of row, :] for rows of `width` dtype elements (zero rows in the padding); dst has rows_max rows.

@@ -298,6 +298,35 @@ route_scatter(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ 
   }
 }
 
+// Routing decision given from outside (a later layer that reuses it): one warp per chunk of 32 tokens counts the
+// chunk's assignments per expert.  Indices outside [0, E) are clamped into range in the working copy idx_ws
+// (so every later table stays in bounds) and reported through the status word.
+__global__ void __launch_bounds__(256)
+idx_chunk_histogram(const int32_t* __restrict__ topk_idx, int32_t* __restrict__ idx_ws, int T_tokens, int E, int K, int n_chunks,
+                    int32_t* __restrict__ chunk_counts, int32_t* __restrict__ status) {
+  const int lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (chunk >= n_chunks) return;
+  const int t = chunk * kChunkTokens + lane;
+  int my_e[kMaxK];
+  bool bad = false;
+  for (int k = 0; k < K; ++k) {
+    int e = -1;
+    if (t < T_tokens) {
+      e = topk_idx[(size_t)t * K + k];
+      if (e < 0 || e >= E) { bad = true; e = min(max(e, 0), E - 1); }
+      idx_ws[(size_t)t * K + k] = e;
+    }
+    my_e[k] = e;
+  }
+  if (bad) atomicExch(status + kStatCode, ROM_ERR_INVALID_ARG);
+  for (int e = 0; e < E; ++e) {
+    int c = 0;
+    for (int k = 0; k < K; ++k) c += __popc(__ballot_sync(0xffffffffu, my_e[k] == e));
+    if (lane == 0) chunk_counts[(size_t)chunk * E + e] = c;
+  }
+}
+
 // One warp per padded row: x_perm[row, :] = x[token(row), :], zeros in padding rows.
 __global__ void __launch_bounds__(256)
 gather_rows(const uint4* __restrict__ x, uint4* __restrict__ x_perm, const int32_t* __restrict__ assign_of_row,
@@ -357,6 +386,9 @@ cudaError_t launch_balance(const rom_config& c, const void* x, const void* W_r, 
   return cudaGetLastError();
 }
 
+static cudaError_t launch_perm_tables(const rom_config& c, const int32_t* idx_ws, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                      int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st);
+
 cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W_r, const float* b_r,
                                int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
                                int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, double* chunk_prob, cudaStream_t st) {
@@ -388,6 +420,15 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
     route_logits_topk<float><<<blocks, threads, smem, st>>>(
         (const float*)x, Wd, b_r, T, c.d_model, c.E, c.K, c.gate_mode, idx_ws, gates, chunk_counts, chunk_prob);
   count_launch();
+  return launch_perm_tables(c, idx_ws, counts, offsets, perm, inv_perm, ws, lay, st);
+}
+
+// offsets, padded offsets, row tiles and the permutation from the per-chunk histogram and the indices
+static cudaError_t launch_perm_tables(const rom_config& c, const int32_t* idx_ws, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                      int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st) {
+  const int T = (int)lay.T;
+  int32_t* chunk_counts = reinterpret_cast<int32_t*>(ws + lay.chunk_counts);
+  int32_t* assign_of_row = reinterpret_cast<int32_t*>(ws + lay.assign_of_row);
   route_offsets<<<1, 1024, 0, st>>>(chunk_counts, (int)lay.n_chunks, c.E,
                                    reinterpret_cast<int32_t*>(ws + lay.counts), reinterpret_cast<int32_t*>(ws + lay.offsets),
                                    reinterpret_cast<int32_t*>(ws + lay.pad_offsets), reinterpret_cast<int32_t*>(ws + lay.num_m_tiles),
@@ -416,6 +457,19 @@ cudaError_t launch_gather_rows_to(const rom_config& c, const void* src, void* ds
                                           (int)lay.rows_max);
   count_launch();
   return cudaGetLastError();
+}
+
+cudaError_t launch_perm_from_idx(const rom_config& c, const int32_t* topk_idx, int32_t* counts, int32_t* offsets, int32_t* perm,
+                                 int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st) {
+  int32_t* idx_ws = reinterpret_cast<int32_t*>(ws + lay.topk_idx);
+  cudaError_t err = cudaMemsetAsync(ws + lay.assign_of_row, 0xff, sizeof(int32_t) * lay.rows_max, st);
+  if (err != cudaSuccess) return err;
+  const int wpb = 8;
+  idx_chunk_histogram<<<((int)lay.n_chunks + wpb - 1) / wpb, wpb * 32, 0, st>>>(
+      topk_idx, idx_ws, (int)lay.T, c.E, c.K, (int)lay.n_chunks, reinterpret_cast<int32_t*>(ws + lay.chunk_counts),
+      reinterpret_cast<int32_t*>(ws + lay.status));
+  count_launch();
+  return launch_perm_tables(c, idx_ws, counts, offsets, perm, inv_perm, ws, lay, st);
 }
 
 }  // namespace rom

@@ -247,3 +247,54 @@ def test_layer_batch_permutation_invariance_on_gpu():
     out2 = g.forward(g.dev["x"][pi].contiguous())
     assert torch.equal(out2, out[pi])
     assert torch.equal(g.counts, counts)
+
+
+# ---------------------------------------------------------------------------------------------- FFN-MoE with shared routing
+def run_ffn(s, d_ff, flags=0, seed=91000, bad_index=False):
+    """Route on the GPU (rom_route), hand idx / gates to rom_ffn_moe_forward, compare with the oracle fed the oracle's own
+    routing of the same inputs (indices are bit-exact, so both sides use the same experts)."""
+    p = synth.make_inputs(s, recipe="unit")
+    tdt = synth.torch_dtype(s)
+    g = torch.Generator().manual_seed(seed)
+    W_gu = (torch.randn((s.E, 2 * d_ff, s.d_model), generator=g) / s.d_model ** 0.5).to(tdt)
+    W_down = (torch.randn((s.E, s.d_model, d_ff), generator=g) / d_ff ** 0.5).to(tdt)
+    r = gpu_route(s, p)
+    cfg = rb.config_from_shape(s, flags=flags)
+    idx = torch.from_numpy(r["idx"]).cuda(); gates = torch.from_numpy(r["gates"]).cuda()
+    if bad_index:
+        idx[0, 0] = s.E + 3
+    ws = torch.empty(rb.ffn_moe_workspace_size(cfg, d_ff), dtype=torch.uint8, device="cuda")
+    out = torch.empty((s.B, s.L, s.d_model), dtype=tdt, device="cuda")
+    rb.rom_ffn_moe_forward(cfg, d_ff, W_gu.cuda(), W_down.cuda(), p["x"].cuda(), idx, gates, out, ws)
+    torch.cuda.synchronize()
+    code = rb.rom_get_status(ws)
+    if bad_index:
+        return code
+    assert code == 0, rb.status_string(code)
+    x = np64(p["x"]).reshape(s.T, s.d_model)
+    o_idx, o_gate, _, _ = O.route(x, np64(p["W_r"]), np64(p["b_r"]), s.K, 0)
+    np.testing.assert_array_equal(r["idx"], o_idx)
+    ref = O.ffn_moe_shared_routing(x, np64(W_gu), np64(W_down), o_idx, o_gate)
+    return assert_close(np64(out).reshape(s.T, s.d_model), ref, TOL[s.dtype], "ffn out")
+
+
+@pytest.mark.parametrize("kw,d_ff", [
+    (dict(), 256),                                               # K = 2, ragged L
+    (dict(E=8, K=1, B=3, L=130), 384),                           # top-1: gate and token order fused into the down projection
+    (dict(E=3, K=3, L=64), 128),
+    (dict(E=4, K=1, B=1, L=1), 128),                             # one token
+    (dict(E=6, K=2, router_bias_scale=4.0, L=513), 256),         # skewed loads, some experts nearly empty
+])
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
+def test_ffn_moe_shared_routing(kw, d_ff, dtype, flags):
+    run_ffn(small_shape(dtype=dtype, **kw), d_ff, flags)
+
+
+def test_ffn_moe_small_bf16_config():
+    s = synth.CONFIGS["small_bf16"]
+    run_ffn(s, 4 * s.d_model)
+
+
+def test_ffn_moe_reports_an_index_out_of_range():
+    code = run_ffn(small_shape(E=4, K=2, L=100), 128, bad_index=True)
+    assert code == -1 and "invalid" in rb.status_string(code)
