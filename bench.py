@@ -185,6 +185,26 @@ def run_stage(args, s):
         esz = 2 if s.dtype == "bf16" else 4
         nbytes = s.T * (4 * s.d_inner * esz + 8 * s.d_state)        # u, Delta, z, y at storage width; B, C fp32
         extra = {"exps": s.T * s.d_inner * s.d_state}
+    elif args.stage == "ffn":
+        # the FFN-MoE that follows a RoM layer and shares its routing (Appendix A.2); hidden width 4 * d_model (assumed: the
+        # paper does not state it); idx / gates come from rom_route on the same x
+        d_ff = 4 * s.d_model
+        p = synth.make_inputs(s.replace(d_inner=64, dt_rank=16))
+        x, W_r = p["x"].to(dev), p["W_r"].to(dev)
+        b_r = None if p["b_r"] is None else p["b_r"].to(dev)
+        tdt = synth.torch_dtype(s)
+        g = torch.Generator().manual_seed(s.seed_base + 900)
+        W_gu = (torch.randn((s.E, 2 * d_ff, s.d_model), generator=g) * 0.02).to(tdt).to(dev)
+        W_down = (torch.randn((s.E, s.d_model, d_ff), generator=g) * 0.02).to(tdt).to(dev)
+        rws = rb.alloc_workspace(cfg, dev)
+        idx = torch.empty((s.T, s.K), dtype=torch.int32, device=dev)
+        gates = torch.empty((s.T, s.K), dtype=torch.float32, device=dev)
+        rb.rom_route(cfg, x, W_r, b_r, idx, gates, None, None, None, None, rws)
+        ws = torch.empty(rb.ffn_moe_workspace_size(cfg, d_ff), dtype=torch.uint8, device=dev)
+        out = torch.empty_like(x)
+        call = lambda: rb.rom_ffn_moe_forward(cfg, d_ff, W_gu, W_down, x, idx, gates, out, ws)
+        nbytes = 2 * s.T * s.d_model * x.element_size() + 3 * s.E * d_ff * s.d_model * x.element_size()
+        extra = {"flops": 6 * s.T * s.K * s.d_model * d_ff, "d_ff": d_ff}
     else:
         p = synth.make_inputs(s.replace(d_inner=64, dt_rank=16))
         x, W_r = p["x"].to(dev), p["W_r"].to(dev)
@@ -208,6 +228,12 @@ def run_stage(args, s):
     line = {"stage": args.stage, "workload": s.name, "ms": ms, "algorithmic_bytes": nbytes,
             "achieved_gbs": nbytes / ms / 1e6, "hbm_peak_gbs": peaks["hbm_gbs"], "frac": nbytes / ms / 1e6 / peaks["hbm_gbs"],
             "peak_source": peaks["source"]}
+    if "flops" in extra:
+        line["d_ff"] = extra["d_ff"]
+        line["tokens_per_s"] = s.T / ms * 1e3
+        line["achieved_tflops"] = extra["flops"] / ms / 1e9
+        line["bf16_peak_tflops"] = peaks["bf16_tflops"]
+        line["tensor_frac"] = line["achieved_tflops"] / peaks["bf16_tflops"]
     if "exps" in extra:
         line["mufu_floor_ms"] = extra["exps"] / (148 * 16 * 1.965e9) * 1e3
         line["mufu_frac"] = line["mufu_floor_ms"] / ms
@@ -232,8 +258,8 @@ def main():
     ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
                     help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
                          "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
-    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route"],
-                    help="layer: the whole forward (the benchmark); scan / route: that entry point alone, timed in isolation "
+    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn"],
+                    help="layer: the whole forward (the benchmark); scan / route / ffn: that entry point alone, timed in isolation "
                          "at the workload's shape (kernel studies and ncu captures; prints a short JSON line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
