@@ -98,22 +98,29 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
   const int ld = 2 * De;
   const size_t tok0 = (size_t)b * L;
 
-  // rows tb-3 .. tb+TCH-1 of H.  K = 1: kept as raw 16-byte words (row indices first, then all rows in
-  // flight at once) and converted on use; K > 1: summed over the slots as they arrive.
+  // rows tb-3 .. tb+TCH-1 of H.  K = 1, 2: kept as raw 16-byte words (row indices first, then all rows in
+  // flight at once), converted and summed over the slots on use; other K: summed over the slots as they arrive.
   constexpr int NR = TCH + 3;
-  RawVec<T> raw[KT == 1 ? NR : 1];
-  float hsum[KT == 1 ? 1 : NR][V];
-  if constexpr (KT == 1) {
-    int32_t rix[NR];
+  constexpr bool RAWP = KT == 1 || KT == 2;
+  constexpr int KS = RAWP ? KT : 1;
+  RawVec<T> raw[RAWP ? NR : 1][KS];
+  int32_t rix[RAWP ? NR : 1][KS];
+  float hsum[RAWP ? 1 : NR][V];
+  if constexpr (RAWP) {
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
       const int t = tb - 3 + r;
-      rix[r] = (t >= 0 && t < L) ? (row_of_assign ? __ldg(row_of_assign + tok0 + t) : (int32_t)(tok0 + t)) : -1;
+#pragma unroll
+      for (int k = 0; k < KS; ++k)
+        rix[r][k] = (t >= 0 && t < L) ? (row_of_assign ? __ldg(row_of_assign + (tok0 + t) * KS + k) : (int32_t)(tok0 + t)) : -1;
     }
 #pragma unroll
     for (int r = 0; r < NR; ++r) {
-      if (rix[r] >= 0) raw[r].load(XZp + (size_t)rix[r] * ld + c0);
-      else raw[r].zero();
+#pragma unroll
+      for (int k = 0; k < KS; ++k) {
+        if (rix[r][k] >= 0) raw[r][k].load(XZp + (size_t)rix[r][k] * ld + c0);
+        else raw[r][k].zero();
+      }
     }
   } else {
 #pragma unroll
@@ -127,8 +134,15 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
     }
   }
   auto hrow = [&](int r, float (&out)[V]) {
-    if constexpr (KT == 1) raw[r].get(out);
-    else {
+    if constexpr (RAWP) {
+      raw[r][0].get(out);
+      if constexpr (KS == 2) {
+        float v2[V];
+        raw[r][1].get(v2);
+#pragma unroll
+        for (int i = 0; i < V; ++i) out[i] += v2[i];
+      }
+    } else {
 #pragma unroll
       for (int i = 0; i < V; ++i) out[i] = hsum[r][i];
     }
@@ -167,15 +181,37 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
   }
   if (Zs != nullptr) {
     // G = SiLU(sum over the selected experts of the Gate Proj rows) (indicator only), one row per token
+    if constexpr (KS == 2) {
+      // the Gate rows of the TCH tokens: same row indices as H, all requested before any is used
 #pragma unroll
-    for (int r = 0; r < TCH; ++r) {
-      const int t = tb + r;
-      if (t >= L) break;
-      float zsum[V];
-      load_sum<T, V, KT>(XZp + De, ld, row_of_assign, K, tok0 + t, c0, zsum);
+      for (int r = 0; r < TCH; ++r) {
 #pragma unroll
-      for (int i = 0; i < V; ++i) zsum[i] = sizeof(T) == 2 ? silu_fast(zsum[i]) : silu_f(zsum[i]);
-      store_vec(Zs + (tok0 + t) * De + c0, zsum);
+        for (int k = 0; k < KS; ++k) {
+          if (rix[r + 3][k] >= 0) raw[r][k].load(XZp + De + (size_t)rix[r + 3][k] * ld + c0);
+          else raw[r][k].zero();
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < TCH; ++r) {
+        const int t = tb + r;
+        if (t >= L) break;
+        float zsum[V];
+        hrow(r, zsum);
+#pragma unroll
+        for (int i = 0; i < V; ++i) zsum[i] = sizeof(T) == 2 ? silu_fast(zsum[i]) : silu_f(zsum[i]);
+        store_vec(Zs + (tok0 + t) * De + c0, zsum);
+      }
+    } else {
+#pragma unroll
+      for (int r = 0; r < TCH; ++r) {
+        const int t = tb + r;
+        if (t >= L) break;
+        float zsum[V];
+        load_sum<T, V, KT>(XZp + De, ld, row_of_assign, K, tok0 + t, c0, zsum);
+#pragma unroll
+        for (int i = 0; i < V; ++i) zsum[i] = sizeof(T) == 2 ? silu_fast(zsum[i]) : silu_f(zsum[i]);
+        store_vec(Zs + (tok0 + t) * De + c0, zsum);
+      }
     }
   }
 }
