@@ -34,7 +34,8 @@ sort, gate sums, tie rule, two-half scan, parameter counts printed in the paper;
 per-expert small projections: E=1 / identical experts reduce to the shared form, rows of
 one expert equal the shared form with that expert's matrices, per-token brute force;
 FFN-MoE with shared routing: library SwiGLU for E=1, per-token loops, identical experts with
-gates summing to one = the dense FFN, linearity in the gates.
+gates summing to one = the dense FFN, linearity in the gates;
+single-token step: a sequence fed token by token reproduces the full-sequence forward and its states.
 """
 from __future__ import annotations
 
@@ -343,6 +344,53 @@ def rom_layer_forward(x, W_r, b_r, W_inz, w_conv, b_conv, W_x, W_dt, b_dt, A, D,
     return out, dict(idx=idx, gate=gate, P=P, logit=logit, counts=counts, offsets=offsets,
                      perm=perm, inv_perm=inv, H=H, Zpre=Zpre, U=U.reshape(T, De), delta=delta,
                      Bm=Bm, Cm=Cm, Delta=Delta, Y=Y.reshape(T, De), Yg=Yg, h_last=h_last)
+
+
+# --------------------------------------------------------------------------- single-token step (recurrent inference)
+def rom_layer_step(x_t, conv_state, ssm_state, W_r, b_r, W_inz, w_conv, b_conv, W_x, W_dt, b_dt, A, D, W_out,
+                   K, dt_rank, gate_mode=0, disc_mode=0):
+    """One token per sequence through the RoM layer with the state carried between calls: the recurrent
+    form of the same equations (Section 3.1: the state-space model as a linear recurrence, which is what
+    gives constant cost per generated token; Section 4.2 routing and expert equations unchanged).
+
+    x_t[B,D_m]: the new token of each sequence.
+    conv_state[B,k-1,D_e]: H of the previous k-1 tokens, oldest first (zeros at a sequence start).
+    ssm_state[B,D_e,N]: h_{t-1} (zeros at a sequence start).
+    Returns out_t[B,D_m], new conv_state, new ssm_state.  Nothing here is shared with the full-sequence
+    functions except the routed projections: the conv tap sum and the state update are written for one step.
+    """
+    x_t = np.asarray(x_t, dtype=F64)
+    conv_state = np.asarray(conv_state, dtype=F64)
+    h = np.array(ssm_state, dtype=F64)
+    A = np.asarray(A, dtype=F64)
+    w = np.asarray(w_conv, dtype=F64)
+    Bsz = x_t.shape[0]
+    k = w.shape[0]
+    N = A.shape[1]
+    idx, gate, _, _ = route(x_t, W_r, b_r, K, gate_mode)
+    H_t, Zpre = expert_in_proj(x_t, W_inz, idx)                       # [B,D_e] each
+    window = np.concatenate([conv_state, H_t[:, None, :]], axis=1)    # [B,k,D_e], oldest first, current last
+    pre = np.zeros_like(H_t)
+    if b_conv is not None:
+        pre = pre + np.asarray(b_conv, dtype=F64)[None, :]
+    for j in range(k):
+        pre = pre + w[j][None, :] * window[:, j, :]
+    U_t = silu(pre)
+    if np.asarray(W_x).ndim == 3:
+        Bm, Cm, Delta = small_proj_routed(U_t, W_x, W_dt, b_dt, idx, dt_rank, N)
+    else:
+        _, Bm, Cm, Delta = small_proj(U_t, W_x, W_dt, b_dt, dt_rank, N)
+    dA = Delta[:, :, None] * A[None, :, :]
+    if disc_mode == 0:
+        Bbar = np.expm1(dA) / A[None, :, :] * Bm[:, None, :]
+    else:
+        Bbar = Delta[:, :, None] * Bm[:, None, :]
+    h = np.exp(dA) * h + Bbar * U_t[:, :, None]
+    Y_t = np.sum(Cm[:, None, :] * h, axis=2)
+    if D is not None:
+        Y_t = Y_t + np.asarray(D, dtype=F64)[None, :] * U_t
+    out_t = expert_out_proj(gated(Y_t, Zpre), W_out, idx, gate)
+    return out_t, window[:, 1:, :].copy(), h
 
 
 # --------------------------------------------------------------------------- FFN-MoE with shared routing

@@ -481,6 +481,44 @@ def test_ffn_moe_identical_experts_and_gate_linearity():
     assert np.abs(O.ffn_moe_shared_routing(x2, W_sw, W_down2, idx2, gate2) - Y2).max() > 1e-3
 
 
+# ---------------------------------------------------------------------------------------------- single-token step
+@pytest.mark.parametrize("K,disc_mode,routed_small", [(1, 0, False), (2, 0, False), (2, 1, False), (1, 0, True)])
+def test_token_by_token_steps_reproduce_the_full_forward(K, disc_mode, routed_small):
+    """Feeding a sequence one token at a time with carried states gives the full-sequence outputs, the last
+    k-1 rows of H as conv state and the full scan's final state (the full forward is pinned above)."""
+    p, s = small_layer(41, B=3, L=9, E=3)
+    if routed_small:
+        g = rng(42)
+        p["W_x"] = g.normal(size=(s["E"],) + p["W_x"].shape) * 0.5
+        p["W_dt"] = g.normal(size=(s["E"],) + p["W_dt"].shape) * 0.5
+    full, im = run_layer(p, K=K, R=s["R"], disc_mode=disc_mode, return_intermediates=True)
+    B, L, De, N, k = s["B"], s["L"], s["De"], s["N"], s["k"]
+    conv_state = np.zeros((B, k - 1, De)); h = np.zeros((B, De, N))
+    for t in range(L):
+        out_t, conv_state, h = O.rom_layer_step(p["x"][:, t], conv_state, h, p["W_r"], p.get("b_r"), p["W_inz"], p["w_conv"],
+                                                p["b_conv"], p["W_x"], p["W_dt"], p["b_dt"], p["A"], p["D"], p["W_out"],
+                                                K=K, dt_rank=s["R"], disc_mode=disc_mode)
+        np.testing.assert_allclose(out_t, full[:, t], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(h, im["h_last"], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(conv_state, im["H"].reshape(B, L, De)[:, L - (k - 1):], rtol=1e-12, atol=1e-14)
+
+
+def test_step_from_given_states_continues_a_split_sequence():
+    """States taken from a full forward over the first part of a sequence continue it exactly."""
+    p, s = small_layer(43, B=2, L=10, E=3)
+    full, im = run_layer(p, K=2, R=s["R"], return_intermediates=True)
+    B, L, De, k = s["B"], s["L"], s["De"], s["k"]
+    cut = 6
+    q = dict(p); q["x"] = p["x"][:, :cut]
+    _, im1 = run_layer(q, K=2, R=s["R"], return_intermediates=True)
+    conv_state = im1["H"].reshape(B, cut, De)[:, cut - (k - 1):]
+    h = im1["h_last"]
+    for t in range(cut, L):
+        out_t, conv_state, h = O.rom_layer_step(p["x"][:, t], conv_state, h, p["W_r"], None, p["W_inz"], p["w_conv"], p["b_conv"],
+                                                p["W_x"], p["W_dt"], p["b_dt"], p["A"], p["D"], p["W_out"], K=2, dt_rank=s["R"])
+        np.testing.assert_allclose(out_t, full[:, t], rtol=1e-10, atol=1e-12)
+
+
 # ---------------------------------------------------------------------------------------------- P11
 def test_wiring_reproduces_paper_parameter_counts():
     rows = [l.split() for l in open(os.path.join(GOLDEN, "paper_param_counts.txt")) if l.strip() and not l.startswith("#")]
