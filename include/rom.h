@@ -166,6 +166,20 @@ ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const
                       int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
                       void *ws, size_t ws_bytes, void *stream);
 
+/* Single-token step of the layer (recurrent inference; Section 3.1: the state-space model is a linear
+ * recurrence, so a generated token costs the same whatever the context length).  Same equations and
+ * routing as rom_layer_forward for one new token per sequence, with the state carried by the caller:
+ *   x, out     : [B, d_model] dtype (cfg->L must be 1)
+ *   conv_state : [B, d_conv-1, d_inner] fp32, in/out: H_t (the summed Conv Proj rows) of the previous
+ *                d_conv-1 tokens, oldest first; zeros at the start of a sequence
+ *   ssm_state  : [B, d_inner, d_state] fp32, in/out: h_{t-1}; zeros at the start of a sequence
+ * Feeding a sequence token by token from zero states reproduces rom_layer_forward on the whole sequence
+ * (up to the rounding of the storage dtype).  topk_idx_out [B,K], gates_out [B,K] may be NULL.
+ * ws: rom_workspace_size(cfg) bytes.                                                               */
+ROM_API int rom_layer_step(const rom_config *cfg, const rom_weights *w, const void *x, float *conv_state,
+                   float *ssm_state, void *out, int32_t *topk_idx_out, float *gates_out,
+                   void *ws, size_t ws_bytes, void *stream);
+
 /* Feed-forward SwiGLU mixture of experts that shares the routing decision of the preceding RoM layer
  * (Appendix A.2, the two equations of the hybrid RoM + FFN-MoE model):
  *   Y_t = sum_i R_i * 1[i in TopK] * f_i(X_t),   f_i(x) = W_down,i ( SiLU(W_gate,i x) * (W_up,i x) )

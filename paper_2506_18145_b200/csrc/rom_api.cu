@@ -208,10 +208,14 @@ const char* const kStageNames[kNumStages] = {"route", "gather", "in_proj", "conv
 
 // ev == nullptr: plain launch sequence.  Otherwise ev[0] is recorded before the first stage and
 // ev[i+1] after stage i (kNumStages + 1 events).
+// conv_state / ssm_state (both or neither): single-token step, L == 1, states read and advanced in place.
 int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
-                       float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream, cudaEvent_t* ev) {
+                       float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream, cudaEvent_t* ev,
+                       float* conv_state = nullptr, float* ssm_state = nullptr) {
   int rc = check_config(cfg, 0);
   if (rc != ROM_OK) return rc;
+  if ((conv_state == nullptr) != (ssm_state == nullptr)) return ROM_ERR_INVALID_ARG;
+  if (conv_state && (cfg->L != 1 || !aligned16(conv_state) || !aligned16(ssm_state))) return ROM_ERR_INVALID_ARG;
   if (!w || !x || !out || !ws) return ROM_ERR_INVALID_ARG;
   if (!w->W_r || !w->W_inz || !w->w_conv || !w->W_x || !w->W_dt || !w->A || !w->W_out) return ROM_ERR_INVALID_ARG;
   const void* ptrs[] = {x, out, ws, w->W_r, w->W_inz, w->w_conv, w->W_x, w->W_dt, w->A, w->W_out};
@@ -262,7 +266,11 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
   ROM_STAGE_DONE();
   // S4: un-permute + sum over selected experts + conv + SiLU
-  ROM_CUDA(launch_conv(c, W + lay.XZp, in_token_order ? nullptr : row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
+  if (conv_state)
+    ROM_CUDA(launch_conv_step(c, W + lay.XZp, in_token_order ? nullptr : row_of_assign, w->w_conv, w->b_conv, conv_state, W + lay.U,
+                              c.K > 1 ? W + lay.Zs : nullptr, st));
+  else
+    ROM_CUDA(launch_conv(c, W + lay.XZp, in_token_order ? nullptr : row_of_assign, w->w_conv, w->b_conv, W + lay.U, c.K > 1 ? W + lay.Zs : nullptr, st));
   ROM_STAGE_DONE();
   if (c.small_proj_experts <= 1) {
     // S5: x Proj -> delta_r | B | C  (shared by all experts)
@@ -292,7 +300,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;
   ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
                        reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, (c.K == 1 && !in_token_order) ? row_of_assign : nullptr,
-                       nullptr, W + lay.Ygp, nullptr, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), true, st));
+                       ssm_state, W + lay.Ygp, ssm_state, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), true, st));
   ROM_STAGE_DONE();
   // S10 + S11.  Tensor path with one expert per token: the epilogue of the grouped Out Proj scales each row by
   // its gate and writes it at its token's position (no intermediate rows, no combine pass).  Otherwise: grouped
@@ -322,6 +330,12 @@ extern "C" {
 int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
                       float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream) {
   return layer_forward_impl(cfg, w, x, out, topk_idx_out, gates_out, counts_out, ws, ws_bytes, stream, nullptr);
+}
+
+int rom_layer_step(const rom_config* cfg, const rom_weights* w, const void* x, float* conv_state, float* ssm_state, void* out,
+                   int32_t* topk_idx_out, float* gates_out, void* ws, size_t ws_bytes, void* stream) {
+  if (!conv_state || !ssm_state) return ROM_ERR_INVALID_ARG;
+  return layer_forward_impl(cfg, w, x, out, topk_idx_out, gates_out, nullptr, ws, ws_bytes, stream, nullptr, conv_state, ssm_state);
 }
 
 int rom_layer_forward_profile(const rom_config* cfg, const rom_weights* w, const void* x, void* out, void* ws, size_t ws_bytes,

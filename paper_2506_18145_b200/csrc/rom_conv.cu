@@ -216,6 +216,61 @@ conv_silu_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_a
   }
 }
 
+// Single-token step of the short convolution: one thread = one 16-byte vector of channels of one sequence.
+// conv_state [B, dconv-1, De] fp32 holds H of the previous dconv-1 tokens, oldest first; it is shifted by one and
+// the new H appended.  Taps are applied in the same order as in conv_silu_kernel (right-aligned into 4 slots).
+template <typename T>
+__global__ void __launch_bounds__(128)
+conv_step_kernel(const T* __restrict__ XZp, const int32_t* __restrict__ row_of_assign, const T* __restrict__ w_conv,
+                 const float* __restrict__ b_conv, float* __restrict__ conv_state, T* __restrict__ U, T* __restrict__ Zs,
+                 int De, int K, int dconv) {
+  constexpr int V = Vec<T>::N;
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * V;
+  if (c0 >= De) return;
+  const size_t b = blockIdx.y;
+  const int ld = 2 * De;
+  float win[4][V];                       // slot 3 = the current token, slots 4-dconv .. 2 = the state rows
+  if (row_of_assign) load_sum<T, V, 0>(XZp, ld, row_of_assign, K, b, c0, win[3]);
+  else load_vec(XZp + b * ld + c0, win[3]);
+  float* st = conv_state + b * (size_t)(dconv - 1) * De + c0;
+#pragma unroll
+  for (int j = 0; j < 3; ++j) {
+    const int src = j - (4 - dconv);     // state row feeding slot j
+#pragma unroll
+    for (int i = 0; i < V; ++i) win[j][i] = src >= 0 ? st[(size_t)src * De + i] : 0.0f;
+  }
+  float u[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) u[i] = b_conv ? b_conv[c0 + i] : 0.0f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int src = j - (4 - dconv);
+    if (src < 0) continue;
+    float w[V];
+    load_vec(w_conv + (size_t)src * De + c0, w);
+#pragma unroll
+    for (int i = 0; i < V; ++i) u[i] = fmaf(w[i], win[j][i], u[i]);
+  }
+#pragma unroll
+  for (int i = 0; i < V; ++i) u[i] = sizeof(T) == 2 ? silu_fast(u[i]) : silu_f(u[i]);
+  store_vec(U + b * De + c0, u);
+  // new state: drop the oldest row, append the current H
+#pragma unroll
+  for (int j = 0; j < 3; ++j) {
+    const int dst = j - (4 - dconv);
+    if (dst < 0) continue;
+#pragma unroll
+    for (int i = 0; i < V; ++i) st[(size_t)dst * De + i] = win[j + 1][i];
+  }
+  if (Zs != nullptr) {
+    float zsum[V];
+    load_sum<T, V, 0>(XZp + De, ld, row_of_assign, K, b, c0, zsum);
+#pragma unroll
+    for (int i = 0; i < V; ++i) zsum[i] = sizeof(T) == 2 ? silu_fast(zsum[i]) : silu_f(zsum[i]);
+    store_vec(Zs + b * De + c0, zsum);
+  }
+}
+
 // out[t, :] = sum_k gates[t,k] * Op[row_of_assign[t*K+k], :], slots added in ascending k.
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -322,6 +377,22 @@ cudaError_t launch_small_combine(const rom_config& c, const float* Bp, const flo
     small_combine_kernel<true><<<blocks, 256, 0, st>>>(Bp, Cp, Dpre, row_of_assign, b_dt, Bm, Cm, Delta, c.d_inner, c.d_state, c.K, total);
   else
     small_combine_kernel<false><<<blocks, 256, 0, st>>>(Bp, Cp, Dpre, row_of_assign, b_dt, Bm, Cm, Delta, c.d_inner, c.d_state, c.K, total);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_conv_step(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
+                             const float* b_conv, float* conv_state, void* U, void* Zs, cudaStream_t st) {
+  const bool bf = c.dtype == ROM_BF16;
+  const int V = bf ? 8 : 4;
+  const int threads = 128;
+  dim3 grid((c.d_inner / V + threads - 1) / threads, c.B);
+  if (bf)
+    conv_step_kernel<__nv_bfloat16><<<grid, threads, 0, st>>>((const __nv_bfloat16*)XZp, row_of_assign, (const __nv_bfloat16*)w_conv, b_conv,
+                                                            conv_state, (__nv_bfloat16*)U, (__nv_bfloat16*)Zs, c.d_inner, c.K, c.d_conv);
+  else
+    conv_step_kernel<float><<<grid, threads, 0, st>>>((const float*)XZp, row_of_assign, (const float*)w_conv, b_conv, conv_state,
+                                                     (float*)U, (float*)Zs, c.d_inner, c.K, c.d_conv);
   count_launch();
   return cudaGetLastError();
 }

@@ -126,6 +126,10 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
 // Zs (K > 1 only): [T, d_inner], SiLU of the Gate Proj rows summed over the K slots.
 cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
                         const float* b_conv, void* U, void* Zs, cudaStream_t st);
+// One token per sequence (L == 1): conv_state [B, d_conv-1, d_inner] fp32 holds H of the previous tokens (oldest first)
+// and is advanced by one token.
+cudaError_t launch_conv_step(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
+                             const float* b_conv, float* conv_state, void* U, void* Zs, cudaStream_t st);
 
 // Scan.  z is a [rows, ldz] matrix; the gate row of token t is z_row[t] (z_row == nullptr: row t).
 // y_rows == nullptr: y is [T, d_inner]; otherwise the output row of token t is written K times, to rows

@@ -298,3 +298,71 @@ def test_ffn_moe_small_bf16_config():
 def test_ffn_moe_reports_an_index_out_of_range():
     code = run_ffn(small_shape(E=4, K=2, L=100), 128, bad_index=True)
     assert code == -1 and "invalid" in rb.status_string(code)
+
+
+# ---------------------------------------------------------------------------------------------- single-token step
+def run_steps(s, n_steps, flags=0, routed_small=False):
+    """Feed the first n_steps tokens of every sequence one at a time through rom_layer_step (states carried on the GPU) and
+    through the oracle's step (states carried in fp64); compare every output and the final states."""
+    p = synth.make_inputs(s, recipe="unit", routed_small=routed_small)
+    tdt = synth.torch_dtype(s)
+    s1 = s.replace(L=1)
+    cfg = rb.config_from_shape(s1, flags=flags, small_proj_experts=s.E if routed_small else 0)
+    dev = {k: (None if v is None else v.cuda().contiguous()) for k, v in p.items()}
+    weights = rb.make_weights(dev)
+    ws = rb.alloc_workspace(cfg, "cuda")
+    conv_state = torch.zeros((s.B, s.d_conv - 1, s.d_inner), dtype=torch.float32, device="cuda")
+    ssm_state = torch.zeros((s.B, s.d_inner, s.d_state), dtype=torch.float32, device="cuda")
+    out = torch.empty((s.B, s.d_model), dtype=tdt, device="cuda")
+    idx = torch.empty((s.B, s.K), dtype=torch.int32, device="cuda")
+    o_conv = np.zeros((s.B, s.d_conv - 1, s.d_inner)); o_h = np.zeros((s.B, s.d_inner, s.d_state))
+    wnames = ("W_r", "b_r", "W_inz", "w_conv", "b_conv", "W_x", "W_dt", "b_dt", "A", "D", "W_out")
+    wn = [np64(p[k]) for k in wnames]
+    tol = TOL[s.dtype]
+    outs = []
+    for t in range(n_steps):
+        x_t = dev["x"][:, t].contiguous()
+        rb.rom_layer_step(cfg, weights, x_t, conv_state, ssm_state, out, idx, None, ws)
+        torch.cuda.synchronize()
+        assert rb.rom_get_status(ws) == 0
+        ref, o_conv, o_h = O.rom_layer_step(np64(p["x"][:, t]), o_conv, o_h, *wn, K=s.K, dt_rank=s.dt_rank)
+        assert_close(np64(out), ref, tol, f"step {t} out")
+        outs.append(out.clone())
+    assert_close(np64(conv_state), o_conv, tol, "conv state")
+    assert_close(np64(ssm_state), o_h, tol, "state-space state")
+    return p, torch.stack(outs, dim=1)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(B=3, L=12, E=4, K=2),
+    dict(B=5, L=12, E=8, K=1),
+    dict(B=2, L=12, E=3, K=3, d_conv=3),
+    dict(B=1, L=12, E=4, K=1, d_conv=2, dt_rank=32),
+])
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
+def test_layer_step_parity(kw, dtype, flags):
+    run_steps(small_shape(dtype=dtype, **kw), 12, flags)
+
+
+def test_layer_step_routed_small_projections():
+    run_steps(small_shape(B=4, L=8, E=4, K=2), 8, routed_small=True)
+
+
+def test_layer_steps_reproduce_the_full_forward_on_gpu():
+    """fp32 path: twelve single-token steps against rom_layer_forward on the same twelve tokens."""
+    s = small_shape(B=3, L=12, E=4, K=2, dtype="f32")
+    p, stepped = run_steps(s, 12)
+    full = GpuLayer(s, p).forward()
+    assert_close(np64(stepped), np64(full), 1e-4, "steps vs full forward")
+
+
+def test_layer_step_rejects_a_sequence_length_other_than_one():
+    s = small_shape(B=2, L=4)
+    cfg = rb.config_from_shape(s)
+    p = synth.make_inputs(s, recipe="unit")
+    dev = {k: (None if v is None else v.cuda().contiguous()) for k, v in p.items()}
+    ws = rb.alloc_workspace(cfg, "cuda")
+    cs = torch.zeros((s.B, s.d_conv - 1, s.d_inner), device="cuda"); hs = torch.zeros((s.B, s.d_inner, s.d_state), device="cuda")
+    out = torch.empty((s.B, s.d_model), dtype=torch.bfloat16, device="cuda")
+    rc = rb.rom_layer_step(cfg, rb.make_weights(dev), dev["x"][:, 0].contiguous(), cs, hs, out, None, None, ws, check=False)
+    assert rc == -1
