@@ -185,6 +185,23 @@ def run_stage(args, s):
         esz = 2 if s.dtype == "bf16" else 4
         nbytes = s.T * (4 * s.d_inner * esz + 8 * s.d_state)        # u, Delta, z, y at storage width; B, C fp32
         extra = {"exps": s.T * s.d_inner * s.d_state}
+    elif args.stage == "step":
+        # single-token step at the workload's widths, 64 sequences generating in lock-step; states stay on the device
+        sb = s.replace(B=64, L=1)
+        cfg = rb.config_from_shape(sb)
+        p = synth.make_inputs(sb)
+        d = {k: (None if v is None else v.to(dev)) for k, v in p.items()}
+        weights = rb.make_weights(d)
+        ws = rb.alloc_workspace(cfg, dev)
+        conv_state = torch.zeros((sb.B, sb.d_conv - 1, sb.d_inner), dtype=torch.float32, device=dev)
+        ssm_state = torch.zeros((sb.B, sb.d_inner, sb.d_state), dtype=torch.float32, device=dev)
+        x_t = d["x"][:, 0].contiguous()
+        out = torch.empty_like(x_t)
+        call = lambda: rb.rom_layer_step(cfg, weights, x_t, conv_state, ssm_state, out, None, None, ws)
+        esz = x_t.element_size()
+        # every expert's projections are read once per step (64 tokens reach all 8 experts), plus the shared small ones
+        nbytes = esz * (3 * s.E * s.d_model * s.d_inner + (2 * s.dt_rank + 2 * s.d_state) * s.d_inner) + 4 * sb.B * s.d_inner * (s.d_state + 3)
+        extra = {"step_batch": sb.B}
     elif args.stage == "ffn":
         # the FFN-MoE that follows a RoM layer and shares its routing (Appendix A.2); hidden width 4 * d_model (assumed: the
         # paper does not state it); idx / gates come from rom_route on the same x
@@ -228,6 +245,9 @@ def run_stage(args, s):
     line = {"stage": args.stage, "workload": s.name, "ms": ms, "algorithmic_bytes": nbytes,
             "achieved_gbs": nbytes / ms / 1e6, "hbm_peak_gbs": peaks["hbm_gbs"], "frac": nbytes / ms / 1e6 / peaks["hbm_gbs"],
             "peak_source": peaks["source"]}
+    if "step_batch" in extra:
+        line["sequences"] = extra["step_batch"]
+        line["tokens_per_s"] = extra["step_batch"] / ms * 1e3
     if "flops" in extra:
         line["d_ff"] = extra["d_ff"]
         line["tokens_per_s"] = s.T / ms * 1e3
@@ -258,8 +278,8 @@ def main():
     ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
                     help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
                          "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
-    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn"],
-                    help="layer: the whole forward (the benchmark); scan / route / ffn: that entry point alone, timed in isolation "
+    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn", "step"],
+                    help="layer: the whole forward (the benchmark); scan / route / ffn / step: that entry point alone, timed in isolation "
                          "at the workload's shape (kernel studies and ncu captures; prints a short JSON line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
