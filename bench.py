@@ -36,10 +36,10 @@ UNIT = "tokens/s"
 # ncu capture, keyed by (stage, workload); None = not captured.  The summaries the figures come from
 # are the text files under profiles/.
 NCU_TRAFFIC_BYTES = {
-    # scan stage = pass 1 (372.7 MB) + pass 2 (660.9 MB) of the chunked scan; profiles/scan_long_ctx.md
-    ("scan", "long_ctx"): 1033.6e6,
+    # scan stage = first launch (395.6 MB) + second launch (612.0 MB) of the chunked scan; profiles/scan_long_ctx.md
+    ("scan", "long_ctx"): 1007.6e6,
     # profiles/in_proj_long_ctx.md
-    ("in_proj", "long_ctx"): 614.4e6,
+    ("in_proj", "long_ctx"): 592.9e6,
 }
 
 
