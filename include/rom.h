@@ -166,6 +166,16 @@ ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const
                       int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
                       void *ws, size_t ws_bytes, void *stream);
 
+/* rom_layer_forward with HOST input and output: enqueues on `stream` the copy of x_host to x_dev, the
+ * forward (x_dev -> out_dev) and the copy of out_dev to out_host, and returns without waiting.
+ *   x_host, out_host : HOST pointers, [B, L, d_model] dtype; page-locked memory makes the copies
+ *                      asynchronous (pageable memory works but serialises with the host)
+ *   x_dev, out_dev   : device staging buffers of the same size, owned by the caller
+ * out_host is valid once the stream has been synchronised.  Calls on different streams with their own
+ * staging buffers and workspaces overlap one call's copies with another's kernels.               */
+ROM_API int rom_layer_forward_host(const rom_config *cfg, const rom_weights *w, const void *x_host, void *out_host,
+                           void *x_dev, void *out_dev, void *ws, size_t ws_bytes, void *stream);
+
 /* Single-token step of the layer (recurrent inference; Section 3.1: the state-space model is a linear
  * recurrence, so a generated token costs the same whatever the context length).  Same equations and
  * routing as rom_layer_forward for one new token per sequence, with the state carried by the caller:

@@ -22,7 +22,7 @@ ROM_OK = 0
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
            "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance",
-           "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step")
+           "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step", "rom_layer_forward_host")
 
 
 class RomConfig(ctypes.Structure):
@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         L.rom_ffn_moe_forward.argtypes = [cfgp, ctypes.c_int32, vp, vp, vp, i32p, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_scan.argtypes = [cfgp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_layer_forward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, i32p, vp, i32p, vp, ctypes.c_size_t, vp]
+        L.rom_layer_forward_host.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, vp, vp, vp, ctypes.c_size_t, vp]
         L.rom_layer_step.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, vp, vp, i32p, vp, vp, ctypes.c_size_t, vp]
         L.rom_workspace_find.argtypes = [cfgp, ctypes.c_char_p, szp, szp]
         L.rom_get_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
@@ -190,6 +191,15 @@ def rom_ffn_moe_forward(cfg, d_ff, W_gu, W_down, x, topk_idx, gates, out, ws, st
                                    _ptr(out), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_ffn_moe_forward")
+    return rc
+
+
+def rom_layer_forward_host(cfg, weights: RomWeights, x_host, out_host, x_dev, out_dev, ws, stream=None, check=True) -> int:
+    """x_host / out_host: CPU tensors (pinned for asynchronous copies); x_dev / out_dev: CUDA staging tensors."""
+    rc = lib().rom_layer_forward_host(ctypes.byref(cfg), ctypes.byref(weights), _ptr(x_host, cuda=False), _ptr(out_host, cuda=False),
+                                      _ptr(x_dev), _ptr(out_dev), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_layer_forward_host")
     return rc
 
 

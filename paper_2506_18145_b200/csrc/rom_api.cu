@@ -332,6 +332,21 @@ int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x
   return layer_forward_impl(cfg, w, x, out, topk_idx_out, gates_out, counts_out, ws, ws_bytes, stream, nullptr);
 }
 
+int rom_layer_forward_host(const rom_config* cfg, const rom_weights* w, const void* x_host, void* out_host, void* x_dev,
+                           void* out_dev, void* ws, size_t ws_bytes, void* stream) {
+  if (!cfg || !x_host || !out_host || !x_dev || !out_dev) return ROM_ERR_INVALID_ARG;
+  int rc = check_config(cfg, 0);
+  if (rc != ROM_OK) return rc;
+  if (!ws || ws_bytes < make_layout(*cfg).total) return ws ? ROM_ERR_WORKSPACE : ROM_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)cfg->B * cfg->L * cfg->d_model * (cfg->dtype == ROM_BF16 ? 2 : 4);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ROM_CUDA(cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, st));
+  rc = layer_forward_impl(cfg, w, x_dev, out_dev, nullptr, nullptr, nullptr, ws, ws_bytes, stream, nullptr);
+  if (rc != ROM_OK) return rc;
+  ROM_CUDA(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
+  return ROM_OK;
+}
+
 int rom_layer_step(const rom_config* cfg, const rom_weights* w, const void* x, float* conv_state, float* ssm_state, void* out,
                    int32_t* topk_idx_out, float* gates_out, void* ws, size_t ws_bytes, void* stream) {
   if (!conv_state || !ssm_state) return ROM_ERR_INVALID_ARG;

@@ -366,3 +366,18 @@ def test_layer_step_rejects_a_sequence_length_other_than_one():
     out = torch.empty((s.B, s.d_model), dtype=torch.bfloat16, device="cuda")
     rc = rb.rom_layer_step(cfg, rb.make_weights(dev), dev["x"][:, 0].contiguous(), cs, hs, out, None, None, ws, check=False)
     assert rc == -1
+
+
+def test_layer_forward_host_matches_the_device_entry_point():
+    """rom_layer_forward_host (pinned host in / out, copies enqueued by the library) gives the device path's bits."""
+    s = small_shape(B=2, L=333, E=4, K=2)
+    p = synth.make_inputs(s, recipe="unit")
+    g = GpuLayer(s, p)
+    ref = g.forward().clone()
+    x_host = p["x"].contiguous().pin_memory()
+    out_host = torch.empty_like(p["x"]).pin_memory()
+    x_dev = torch.empty_like(g.dev["x"]); out_dev = torch.empty_like(g.dev["x"])
+    rb.rom_layer_forward_host(g.cfg, g.weights, x_host, out_host, x_dev, out_dev, g.ws)
+    torch.cuda.synchronize()
+    assert rb.rom_get_status(g.ws) == 0
+    assert torch.equal(out_host, ref.cpu())
