@@ -381,3 +381,38 @@ def test_layer_forward_host_matches_the_device_entry_point():
     torch.cuda.synchronize()
     assert rb.rom_get_status(g.ws) == 0
     assert torch.equal(out_host, ref.cpu())
+
+
+# ---------------------------------------------------------------------------------------------- ragged widths, size limits
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
+@pytest.mark.parametrize("kw", [
+    dict(d_model=192, d_inner=320, dt_rank=48, E=5, K=2, B=2, L=257),      # widths that are multiples of 64 only
+    dict(d_model=64, d_inner=64, dt_rank=16, E=2, K=1, B=1, L=700),        # the smallest widths
+    dict(d_model=128, d_inner=192, dt_rank=16, E=64, K=8, B=1, L=300),     # the largest expert count and top-K
+])
+def test_layer_ragged_widths_and_limits(kw, dtype, flags):
+    check_layer(small_shape(dtype=dtype, **kw), "unit", flags=flags)
+
+
+def test_scan_many_short_sequences():
+    """Many sequences of a few steps each: one block per (sequence, channel group), tiles mostly empty."""
+    y, Y, hl, HL = run_scan(B=700, L=5, De=128, dtype="bf16", disc_mode=0, with_z=True, with_h0=True, with_D=True, seed=99100)
+    assert_close(y, Y, TOL["bf16"], "scan y"); assert_close(hl, HL, 2e-3, "scan h_last")
+    y, Y, hl, HL = run_scan(B=3, L=1, De=64, dtype="f32", disc_mode=1, with_z=False, with_h0=False, with_D=False, seed=99200)
+    assert_close(y, Y, 1e-4, "scan y"); assert_close(hl, HL, 1e-4, "scan h_last")
+
+
+def test_argument_errors_launch_nothing():
+    s = small_shape()
+    p = synth.make_inputs(s, recipe="unit")
+    g = GpuLayer(s, p)
+    bad = rb.config_from_shape(s)
+    bad.K = s.E + 1
+    assert rb.rom_layer_forward(bad, g.weights, g.dev["x"], g.out, None, None, None, g.ws, check=False) == -1
+    bad = rb.config_from_shape(s); bad.d_state = 8
+    assert rb.rom_layer_forward(bad, g.weights, g.dev["x"], g.out, None, None, None, g.ws, check=False) == -2
+    bad = rb.config_from_shape(s); bad.small_proj_experts = 3
+    assert rb.rom_layer_forward(bad, g.weights, g.dev["x"], g.out, None, None, None, g.ws, check=False) == -1
+    small_ws = g.ws[:1024]
+    assert rb.rom_layer_forward(g.cfg, g.weights, g.dev["x"], g.out, None, None, None, small_ws, check=False) == -3
+    g.forward()                                       # nothing was enqueued by the rejected calls; the layer still runs
