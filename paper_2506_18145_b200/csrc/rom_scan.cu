@@ -397,6 +397,64 @@ scan_kernel(const ScanArgs p) {
   }
 }
 
+// One step per sequence (L == 1, recurrent inference): a thread owns all 16 states of one channel of one
+// sequence; the state is read and written once (64 contiguous bytes per thread), B and C of the sequence are the
+// same for every thread of the block.  Same arithmetic as scan_kernel (per PRECISE / ZOH).
+template <typename T, bool PRECISE, bool ZOH>
+__global__ void __launch_bounds__(BLOCK)
+scan_step_kernel(const ScanArgs p) {
+  const int c = blockIdx.x * BLOCK + threadIdx.x;
+  const size_t b = blockIdx.y;
+  if (c >= p.De) return;
+  const T* __restrict__ u = static_cast<const T*>(p.u);
+  const float dl = p.delta[b * p.De + c];
+  const float uu = to_f32(u[b * p.De + c]);
+  const float4* Bq = reinterpret_cast<const float4*>(p.Bm + b * NST);
+  const float4* Cq = reinterpret_cast<const float4*>(p.Cm + b * NST);
+  const float4* Aq = reinterpret_cast<const float4*>(p.A + (size_t)c * NST);
+  const float4* Hq = p.h0 ? reinterpret_cast<const float4*>(p.h0 + (b * p.De + c) * NST) : nullptr;
+  float4* Ho = p.h_last ? reinterpret_cast<float4*>(p.h_last + (b * p.De + c) * NST) : nullptr;
+  float y = 0.0f;
+#pragma unroll
+  for (int q = 0; q < NST / 4; ++q) {
+    const float4 a4 = __ldg(Aq + q), b4 = __ldg(Bq + q), c4 = __ldg(Cq + q);
+    const float4 h4 = Hq ? Hq[q] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    const float av[4] = {a4.x, a4.y, a4.z, a4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w}, cv[4] = {c4.x, c4.y, c4.z, c4.w};
+    float hv[4] = {h4.x, h4.y, h4.z, h4.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (PRECISE) {
+        const float dA = dl * av[i];
+        const float w = ZOH ? -expm1f(dA) * (-1.0f / av[i]) * bv[i] * uu : bv[i] * (dl * uu);
+        hv[i] = fmaf(expf(dA), hv[i], w);
+      } else {
+        const float a = ex2_approx(dl * (av[i] * kLog2e));
+        if (ZOH) {
+          const float w = (uu * (-1.0f / av[i])) * bv[i];
+          hv[i] = fmaf(a, hv[i] - w, w);
+        } else {
+          hv[i] = fmaf(a, hv[i], (dl * uu) * bv[i]);
+        }
+      }
+      y = fmaf(cv[i], hv[i], y);
+    }
+    if (Ho) Ho[q] = make_float4(hv[0], hv[1], hv[2], hv[3]);
+  }
+  if (p.D) y = fmaf(p.D[c], uu, y);
+  if (p.z) {
+    const T* __restrict__ z = static_cast<const T*>(p.z);
+    const size_t zrow = p.z_row ? (size_t)__ldg(p.z_row + b) : b;
+    const float zz = to_f32(z[zrow * p.ldz + c]);
+    y *= p.gate_activated ? zz : (PRECISE ? zz / (1.0f + expf(-zz)) : silu_fast(zz));
+  }
+  T* __restrict__ yo = static_cast<T*>(p.y);
+  if (p.y_rows == nullptr) {
+    yo[b * p.De + c] = from_f32<T>(y);
+  } else {
+    for (int kk = 0; kk < p.K; ++kk) yo[(size_t)__ldg(p.y_rows + b * p.K + kk) * p.De + c] = from_f32<T>(y);
+  }
+}
+
 // Initial state of every chunk after the first.  h_end[0] is the true state after chunk 0 (it ran from the
 // caller's h0); for j >= 1, h_end[j] is chunk j's end state from a zero start.  In chunk order, per
 // (sequence, channel, state):  h = h_end[0];  h_in[j] = h;  h = exp(A * sum_delta[j]) * h + h_end[j].
@@ -460,6 +518,14 @@ template <typename T, bool PRECISE>
 cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const float* h0, float* h_last,
                           float* chunk_ws, int num_sms, cudaStream_t st) {
   const bool zoh = c.disc_mode == 0;
+  if (c.L == 1) {
+    a.h0 = h0; a.h_last = h_last;
+    dim3 grid((c.d_inner + BLOCK - 1) / BLOCK, c.B);
+    if (zoh) scan_step_kernel<T, PRECISE, true><<<grid, BLOCK, 0, st>>>(a);
+    else scan_step_kernel<T, PRECISE, false><<<grid, BLOCK, 0, st>>>(a);
+    count_launch();
+    return cudaGetLastError();
+  }
   const int nch = chunk_ws ? scan_chunks(c.B, c.d_inner, c.L) : 1;
   if (nch == 1) {
     a.Lc = c.L; a.L0 = c.L; a.nch = 1;
