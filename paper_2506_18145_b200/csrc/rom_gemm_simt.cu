@@ -51,15 +51,29 @@ gemm_simt(const T* __restrict__ A, int lda, const T* __restrict__ Bw, int ldb, i
   const int tid = threadIdx.x;
   const int ty = tid / 16, tx = tid % 16;
   float acc[4][4] = {};
-  for (int k0 = 0; k0 < Kd; k0 += BK) {
-    for (int i = tid; i < BM * BK; i += 256) {
+  // each thread brings 4 elements of the A tile and 4 of the B tile per K block; the next block's elements are
+  // requested before the current block is multiplied, so the global-memory latency overlaps the arithmetic
+  float pa[4], pb[4];
+  auto fetch = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + 256 * j;
       const int r = i / BK, k = i % BK;
-      const int m = m0 + r, kk = k0 + k;
-      As[k][r] = (m < M && kk < Kd) ? to_f32(A[(size_t)m * lda + kk]) : 0.0f;
-      const int n = n0 + r;
-      Bs[k][r] = (n < N && kk < Kd) ? to_f32(Bp[(size_t)n * ldb + kk]) : 0.0f;
+      const int m = m0 + r, n = n0 + r, kk = k0 + k;
+      pa[j] = (m < M && kk < Kd) ? to_f32(A[(size_t)m * lda + kk]) : 0.0f;
+      pb[j] = (n < N && kk < Kd) ? to_f32(Bp[(size_t)n * ldb + kk]) : 0.0f;
+    }
+  };
+  fetch(0);
+  for (int k0 = 0; k0 < Kd; k0 += BK) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = tid + 256 * j;
+      As[i % BK][i / BK] = pa[j];
+      Bs[i % BK][i / BK] = pb[j];
     }
     __syncthreads();
+    if (k0 + BK < Kd) fetch(k0 + BK);
 #pragma unroll
     for (int k = 0; k < BK; ++k) {
       float a[4], b[4];
