@@ -347,6 +347,19 @@ def main():
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else None
 
+    # ---- per-stage device times (CUDA events between the kernels, same stream, same inputs)
+    stage_ms = {}
+    if rank == 0:
+        acc = {}
+        n_prof = max(3, min(args.steps, 10))
+        for _ in range(n_prof):
+            for k, v in rb.rom_layer_forward_profile(cfg, weights, x_dev, out, ws, stream).items():
+                acc.setdefault(k, []).append(v)
+        stage_ms = {k: sum(v) / len(v) for k, v in acc.items()}
+    code = rb.rom_get_status(ws)
+    if code != 0:
+        raise SystemExit("device status: " + rb.status_string(code))
+
     # ---- end to end: rom_layer_forward_host on pinned HOST buffers; every step copies its x to the device and its
     # out back inside the timed region.  Steps rotate over four streams, each with its own staging buffers and
     # workspace, so one step's copies overlap the others' kernels (input prefetch / output drain of a serving loop).
@@ -384,19 +397,6 @@ def main():
     del lanes
 
     ms, ms_e2e = replicas.max_over_ranks([ms, ms_e2e], dist, dev)
-
-    # ---- per-stage device times (CUDA events between the kernels, same stream, same inputs)
-    stage_ms = {}
-    if rank == 0:
-        acc = {}
-        n_prof = max(3, min(args.steps, 10))
-        for _ in range(n_prof):
-            for k, v in rb.rom_layer_forward_profile(cfg, weights, x_dev, out, ws, stream).items():
-                acc.setdefault(k, []).append(v)
-        stage_ms = {k: sum(v) / len(v) for k, v in acc.items()}
-    code = rb.rom_get_status(ws)
-    if code != 0:
-        raise SystemExit("device status: " + rb.status_string(code))
 
     if rank == 0:
         peaks = load_peaks()

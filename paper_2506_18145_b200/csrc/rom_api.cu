@@ -41,7 +41,7 @@ WsLayout make_layout(const rom_config& c) {
   l.delta_r = take(l.esz * (size_t)l.T * R);
   l.Bm = take(sizeof(float) * (size_t)l.T * N);
   l.Cm = take(sizeof(float) * (size_t)l.T * N);
-  l.Delta = take(sizeof(float) * (size_t)l.T * c.d_inner);
+  l.Delta = take(l.esz * (size_t)l.T * c.d_inner);
   l.Ygp = take(l.esz * (size_t)l.rows_max * c.d_inner);
   l.Op = take(l.esz * (size_t)l.rows_max * c.d_model);
   l.scan_ws = take(sizeof(float) * scan_ws_floats(c.B, c.d_inner, c.L));
@@ -132,7 +132,7 @@ int rom_workspace_find(const rom_config* cfg, const char* name, size_t* offset, 
       {"delta_r", l.delta_r, l.esz * (size_t)l.T * cfg->dt_rank},
       {"Bm", l.Bm, sizeof(float) * (size_t)l.T * cfg->d_state},
       {"Cm", l.Cm, sizeof(float) * (size_t)l.T * cfg->d_state},
-      {"Delta", l.Delta, sizeof(float) * (size_t)l.T * cfg->d_inner},
+      {"Delta", l.Delta, l.esz * (size_t)l.T * cfg->d_inner},
       {"row_of_assign", l.row_of_assign, sizeof(int32_t) * (size_t)l.A},
       {"XZp", l.XZp, l.esz * (size_t)l.rows_max * 2 * cfg->d_inner},
       {"Ygp", l.Ygp, l.esz * (size_t)l.rows_max * cfg->d_inner},
@@ -194,7 +194,7 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
     if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
     chunk_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + lay.scan_ws);
   }
-  ROM_CUDA(launch_scan(*cfg, u, delta, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, chunk_ws, false, st));
+  ROM_CUDA(launch_scan(*cfg, u, delta, true, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, chunk_ws, false, st));
   return ROM_OK;
 }
 
@@ -292,13 +292,13 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
     ROM_CUDA(gemm(W + lay.delta_rp, R, w->W_dt, R, c.E, (int64_t)De * R, (int)lay.rows_max, De, R, tile_expert, num_m_tiles, e_dt));
     ROM_CUDA(launch_small_combine(c, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp),
                                   reinterpret_cast<float*>(W + lay.Dpre), row_of_assign, w->b_dt, reinterpret_cast<float*>(W + lay.Bm),
-                                  reinterpret_cast<float*>(W + lay.Cm), reinterpret_cast<float*>(W + lay.Delta), st));
+                                  reinterpret_cast<float*>(W + lay.Cm), W + lay.Delta, st));
     ROM_STAGE_DONE();
   }
   // S7 + S8 + S9: scan, gate, re-permute
   // K = 1: the gate row of a token is its Gate Proj row in expert order; K > 1: the summed rows from S4
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;
-  ROM_CUDA(launch_scan(c, W + lay.U, reinterpret_cast<float*>(W + lay.Delta), w->A, reinterpret_cast<float*>(W + lay.Bm),
+  ROM_CUDA(launch_scan(c, W + lay.U, W + lay.Delta, false, w->A, reinterpret_cast<float*>(W + lay.Bm),
                        reinterpret_cast<float*>(W + lay.Cm), w->D, zbase, c.K == 1 ? 2 * De : De, (c.K == 1 && !in_token_order) ? row_of_assign : nullptr,
                        ssm_state, W + lay.Ygp, ssm_state, row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), true, st));
   ROM_STAGE_DONE();

@@ -298,18 +298,19 @@ combine_kernel(const T* __restrict__ Op, const int32_t* __restrict__ row_of_assi
 
 // Per-expert x Proj / dt Proj: one thread per float4 of a token's [Delta | B | C] row; the K slots are added in
 // ascending order, then (Delta only) the shared bias and the softplus.
-template <bool PRECISE>
+template <typename T>
 __global__ void __launch_bounds__(256)
 small_combine_kernel(const float* __restrict__ Bp, const float* __restrict__ Cp, const float* __restrict__ Dpre,
                      const int32_t* __restrict__ row_of_assign, const float* __restrict__ b_dt, float* __restrict__ Bm,
-                     float* __restrict__ Cm, float* __restrict__ Delta, int De, int N, int K, long long total_vec) {
+                     float* __restrict__ Cm, T* __restrict__ Delta, int De, int N, int K, long long total_vec) {
+  constexpr bool PRECISE = sizeof(T) == 4;
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total_vec) return;
   const int vpr = (De + 2 * N) / 4;
   const long long t = i / vpr;
   const int c0 = (int)(i % vpr) * 4;
-  const float* src; float* dst; int ld, col;
-  if (c0 < De) { src = Dpre; dst = Delta; ld = De; col = c0; }
+  const float* src; float* dst = nullptr; int ld, col;
+  if (c0 < De) { src = Dpre; ld = De; col = c0; }
   else if (c0 < De + N) { src = Bp; dst = Bm; ld = N; col = c0 - De; }
   else { src = Cp; dst = Cm; ld = N; col = c0 - De - N; }
   float4 acc = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
@@ -322,6 +323,9 @@ small_combine_kernel(const float* __restrict__ Bp, const float* __restrict__ Cp,
     const float4 b = b_dt ? __ldg(reinterpret_cast<const float4*>(b_dt + col)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     if (PRECISE) acc = make_float4(softplus_f(acc.x + b.x), softplus_f(acc.y + b.y), softplus_f(acc.z + b.z), softplus_f(acc.w + b.w));
     else acc = make_float4(softplus_fast(acc.x + b.x), softplus_fast(acc.y + b.y), softplus_fast(acc.z + b.z), softplus_fast(acc.w + b.w));
+    T* d = Delta + (size_t)t * ld + col;
+    d[0] = from_f32<T>(acc.x); d[1] = from_f32<T>(acc.y); d[2] = from_f32<T>(acc.z); d[3] = from_f32<T>(acc.w);
+    return;
   }
   *reinterpret_cast<float4*>(dst + (size_t)t * ld + col) = acc;
 }
@@ -369,14 +373,14 @@ cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* r
 }
 
 cudaError_t launch_small_combine(const rom_config& c, const float* Bp, const float* Cp, const float* Dpre,
-                                 const int32_t* row_of_assign, const float* b_dt, float* Bm, float* Cm, float* Delta,
+                                 const int32_t* row_of_assign, const float* b_dt, float* Bm, float* Cm, void* Delta,
                                  cudaStream_t st) {
   const long long total = (long long)c.B * c.L * ((c.d_inner + 2 * c.d_state) / 4);
   const unsigned blocks = (unsigned)((total + 255) / 256);
   if (c.dtype == ROM_F32)
-    small_combine_kernel<true><<<blocks, 256, 0, st>>>(Bp, Cp, Dpre, row_of_assign, b_dt, Bm, Cm, Delta, c.d_inner, c.d_state, c.K, total);
+    small_combine_kernel<float><<<blocks, 256, 0, st>>>(Bp, Cp, Dpre, row_of_assign, b_dt, Bm, Cm, (float*)Delta, c.d_inner, c.d_state, c.K, total);
   else
-    small_combine_kernel<false><<<blocks, 256, 0, st>>>(Bp, Cp, Dpre, row_of_assign, b_dt, Bm, Cm, Delta, c.d_inner, c.d_state, c.K, total);
+    small_combine_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(Bp, Cp, Dpre, row_of_assign, b_dt, Bm, Cm, (__nv_bfloat16*)Delta, c.d_inner, c.d_state, c.K, total);
   count_launch();
   return cudaGetLastError();
 }

@@ -26,7 +26,7 @@ __device__ __forceinline__ void epi_store_scalar(const Epilogue& ep, int m, int 
       reinterpret_cast<float*>(ep.C)[(size_t)m * ep.ldc + n] = v;
       break;
     default:
-      reinterpret_cast<float*>(ep.C)[(size_t)m * ep.ldc + n] = softplus_f(v + (ep.bias ? ep.bias[n] : 0.0f));
+      reinterpret_cast<T*>(ep.C)[(size_t)m * ep.ldc + n] = from_f32<T>(softplus_f(v + (ep.bias ? ep.bias[n] : 0.0f)));
       break;
   }
 }

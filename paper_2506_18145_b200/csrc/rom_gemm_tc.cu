@@ -175,12 +175,7 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
       *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
       *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
     } else {
-      const float4 b0 = bq[j / 4], b1 = bq[j / 4 + 1];
-      float* dst = reinterpret_cast<float*>(ep.C) + m * ep.ldc + n;
-      *reinterpret_cast<float4*>(dst) = make_float4(softplus_fast(v[0] + b0.x), softplus_fast(v[1] + b0.y),
-                                                    softplus_fast(v[2] + b0.z), softplus_fast(v[3] + b0.w));
-      *reinterpret_cast<float4*>(dst + 4) = make_float4(softplus_fast(v[4] + b1.x), softplus_fast(v[5] + b1.y),
-                                                        softplus_fast(v[6] + b1.z), softplus_fast(v[7] + b1.w));
+      // (softplus and plain-fp32 output go through epi_softplus32; nothing reaches this branch)
     }
   }
 }
@@ -204,13 +199,32 @@ __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, in
     *reinterpret_cast<float4*>(sw + lane * 32 + ((c ^ (lane & 7)) << 2)) = o;
   }
   __syncwarp();
-  const int c = lane & 7;
-  const int n = n0 + 4 * c;
+  if constexpr (MODE == EPI_F32) {
+    const int c = lane & 7;
+    const int n = n0 + 4 * c;
 #pragma unroll
-  for (int r4 = 0; r4 < 8; ++r4) {
-    const int R = r4 * 4 + (lane >> 3);
-    const float4 v = *reinterpret_cast<const float4*>(sw + R * 32 + ((c ^ (R & 7)) << 2));
-    if (row0 + R < M_valid && n < N) *reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.C) + (size_t)(row0 + R) * ep.ldc + n) = v;
+    for (int r4 = 0; r4 < 8; ++r4) {
+      const int R = r4 * 4 + (lane >> 3);
+      const float4 v = *reinterpret_cast<const float4*>(sw + R * 32 + ((c ^ (R & 7)) << 2));
+      if (row0 + R < M_valid && n < N) *reinterpret_cast<float4*>(reinterpret_cast<float*>(ep.C) + (size_t)(row0 + R) * ep.ldc + n) = v;
+    }
+  } else {
+    // rounded to bf16: a lane takes 8 columns (two staged float4), 4 lanes one 64-byte row segment, 8 rows per store
+    const int c8 = lane & 3;
+    const int n = n0 + 8 * c8;
+#pragma unroll
+    for (int r8 = 0; r8 < 4; ++r8) {
+      const int R = r8 * 8 + (lane >> 2);
+      const float4 v0 = *reinterpret_cast<const float4*>(sw + R * 32 + (((2 * c8) ^ (R & 7)) << 2));
+      const float4 v1 = *reinterpret_cast<const float4*>(sw + R * 32 + (((2 * c8 + 1) ^ (R & 7)) << 2));
+      uint4 q;
+      __nv_bfloat162 h0 = __floats2bfloat162_rn(v0.x, v0.y), h1 = __floats2bfloat162_rn(v0.z, v0.w);
+      __nv_bfloat162 h2 = __floats2bfloat162_rn(v1.x, v1.y), h3 = __floats2bfloat162_rn(v1.z, v1.w);
+      q.x = *reinterpret_cast<uint32_t*>(&h0); q.y = *reinterpret_cast<uint32_t*>(&h1);
+      q.z = *reinterpret_cast<uint32_t*>(&h2); q.w = *reinterpret_cast<uint32_t*>(&h3);
+      if (row0 + R < M_valid && n < N)
+        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + (size_t)(row0 + R) * ep.ldc + n) = q;
+    }
   }
   __syncwarp();
 }

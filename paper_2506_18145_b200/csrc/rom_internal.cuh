@@ -63,7 +63,7 @@ inline void count_launch() { LaunchCounter::count++; }
 enum EpiMode : int {
   EPI_STORE = 0,      // C[m, n] = acc                          (dtype)
   EPI_XPROJ = 1,      // n < R: delta_r[m, n] (dtype); then Bm[m, n-R], Cm[m, n-R-N] (fp32)
-  EPI_SOFTPLUS = 2,   // Delta[m, n] = softplus(acc + bias[n])  (fp32)
+  EPI_SOFTPLUS = 2,   // Delta[m, n] = softplus(acc + bias[n])  (dtype)
   EPI_INPROJ = 3,     // C[m, n] = acc for n < R (Conv Proj), SiLU(acc) for n >= R (Gate Proj)   (dtype); with row_token
                       // (tensor path, top-1) row m is written at row row_token[m], i.e. back in token order
   EPI_OUTPROJ = 4,    // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
@@ -74,7 +74,7 @@ enum EpiMode : int {
 };
 struct Epilogue {
   int mode;
-  void* C;            // EPI_STORE: [M, ldc] dtype;  EPI_XPROJ: delta_r [M, R] dtype;  EPI_SOFTPLUS: float [M, ldc]
+  void* C;            // EPI_STORE, EPI_SOFTPLUS: [M, ldc] dtype;  EPI_XPROJ: delta_r [M, R] dtype;  EPI_F32: float [M, ldc]
   int ldc;
   float* Bm;          // EPI_XPROJ
   float* Cm;
@@ -109,7 +109,7 @@ cudaError_t launch_gather_rows_to(const rom_config& c, const void* src, void* ds
 // Per-expert x Proj / dt Proj: sums over the K slots of a token, in ascending slot order (fp32):
 //   Bm[t, :] = sum_k Bp[row(t,k), :],  Cm likewise,  Delta[t, c] = softplus(b_dt[c] + sum_k Dpre[row(t,k), c]).
 cudaError_t launch_small_combine(const rom_config& c, const float* Bp, const float* Cp, const float* Dpre,
-                                 const int32_t* row_of_assign, const float* b_dt, float* Bm, float* Cm, float* Delta,
+                                 const int32_t* row_of_assign, const float* b_dt, float* Bm, float* Cm, void* Delta /*dtype*/,
                                  cudaStream_t st);
 
 // C[M,N] = A[M,Kd] * B[e][N,Kd]^T, A and B K-contiguous.  Grouped when tile_expert != nullptr: row tile
@@ -137,7 +137,8 @@ cudaError_t launch_conv_step(const rom_config& c, const void* XZp, const int32_t
 // gate_activated: z already holds SiLU of the gate pre-activation (the producer applied it).
 // chunk_ws == nullptr: one pass per sequence.  Otherwise a long sequence with too few channels to fill the GPU
 // is cut into scan_chunks() chunks scanned in parallel (two passes); chunk_ws holds scan_ws_floats() floats.
-cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
+// delta: [B, L, d_inner], fp32 when delta_fp32, else in the storage dtype.
+cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
                         void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st);
 

@@ -113,7 +113,7 @@ struct Tile {
 };
 
 struct ScanArgs {
-  const void* u; const float* delta; const float* A; const float* Bm; const float* Cm; const float* D;
+  const void* u; const void* delta; const float* A; const float* Bm; const float* Cm; const float* D;
   const void* z; int ldz; const int32_t* z_row; const float* h0; void* y; float* h_last; const int32_t* y_rows;
   int K, L, De;
   int Lc, nch;          // chunk length and chunks per sequence (nch == 1: Lc == L); blockIdx.z = chunk
@@ -122,6 +122,7 @@ struct ScanArgs {
   int gate_activated;   // z already holds SiLU(gate pre-activation): multiply only
   int chunk_off;        // chunk of blockIdx.z == 0
 };
+// TD: type Delta is stored in: float (the rom_scan entry point, the fp32 layer) or the storage type (bf16 layer).
 
 // PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance); otherwise one ex2.approx per
 // state update (bf16 configurations, 2e-2 tolerance).
@@ -129,7 +130,7 @@ struct ScanArgs {
 // MODE 0: full scan.  MODE 1: state only (no outputs, only h_last and sum_delta of every chunk).  MODE 2: first
 // launch of the chunked scan: chunk 0 runs the full scan from the caller's initial state (h0 indexed by
 // sequence), the other chunks run state-only from a zero state.
-template <typename T, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
+template <typename T, typename TD, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
 __global__ void __launch_bounds__(BLOCK, NS >= 8 ? 2 : 1)
 scan_kernel(const ScanArgs p) {
   using G = Geo<NC, NS>;
@@ -186,14 +187,14 @@ scan_kernel(const ScanArgs p) {
 #pragma unroll
   for (int i = 0; i < 8; ++i) dsk[i] = p.D ? p.D[lc_eff + i] : 0.0f;
   // running pointers to this thread's piece of the next tile to fetch
-  const float* dptr = p.delta + (tok0 + lr) * De + lc_eff;
+  const TD* dptr = static_cast<const TD*>(p.delta) + (tok0 + lr) * De + lc_eff;
   const T* uptr = u + (tok0 + lr) * De + lc_eff;
   const size_t row_step = (size_t)TS * De;
   // B/C: word i of this thread is element (r = warp + 8 i, j = lane) of the [TS][32] tile (B | C)
   const float* bcptr = (lane < NST ? p.Bm : p.Cm) + (tok0 + warp) * NST + (lane & 15);
   const int bc_dst = ((lane & 15) >> 1) * 4 + ((lane >> 4) << 1) + (lane & 1);
 
-  Raw8<float> pre_d;
+  Raw8<TD> pre_d;
   Raw8<T> pre_u, pre_z, cur_u, cur_z;
   float pre_bc[G::NBC];
 
@@ -400,14 +401,14 @@ scan_kernel(const ScanArgs p) {
 // One step per sequence (L == 1, recurrent inference): a thread owns all 16 states of one channel of one
 // sequence; the state is read and written once (64 contiguous bytes per thread), B and C of the sequence are the
 // same for every thread of the block.  Same arithmetic as scan_kernel (per PRECISE / ZOH).
-template <typename T, bool PRECISE, bool ZOH>
+template <typename T, typename TD, bool PRECISE, bool ZOH>
 __global__ void __launch_bounds__(BLOCK)
 scan_step_kernel(const ScanArgs p) {
   const int c = blockIdx.x * BLOCK + threadIdx.x;
   const size_t b = blockIdx.y;
   if (c >= p.De) return;
   const T* __restrict__ u = static_cast<const T*>(p.u);
-  const float dl = p.delta[b * p.De + c];
+  const float dl = to_f32(static_cast<const TD*>(p.delta)[b * p.De + c]);
   const float uu = to_f32(u[b * p.De + c]);
   const float4* Bq = reinterpret_cast<const float4*>(p.Bm + b * NST);
   const float4* Cq = reinterpret_cast<const float4*>(p.Cm + b * NST);
@@ -476,14 +477,14 @@ chain_chunk_states(const float* __restrict__ A, const float* __restrict__ h_end,
   if (h_last) h_last[i] = h;
 }
 
-template <typename T, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
+template <typename T, typename TD, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
 cudaError_t launch_one(const ScanArgs& a, int B, int grid_z, cudaStream_t st) {
   using G = Geo<NC, NS>;
   const size_t smem = 2 * sizeof(Tile<NC, NS>) + (2 * (size_t)G::TS * G::YP + (BLOCK / 32) * G::STRIP) * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, NC, NS, PRECISE, ZOH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = cudaFuncSetAttribute(scan_kernel<T, TD, NC, NS, PRECISE, ZOH, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((a.De + G::CH - 1) / G::CH, B, grid_z);
-  scan_kernel<T, NC, NS, PRECISE, ZOH, MODE><<<grid, BLOCK, smem, st>>>(a);
+  scan_kernel<T, TD, NC, NS, PRECISE, ZOH, MODE><<<grid, BLOCK, smem, st>>>(a);
   count_launch();
   return cudaGetLastError();
 }
@@ -503,26 +504,26 @@ int pick_thread_shape(int B, int De, int num_sms) {
   return 102;
 }
 
-template <typename T, bool PRECISE, bool ZOH>
+template <typename T, typename TD, bool PRECISE, bool ZOH>
 cudaError_t launch_shape(int shape, const ScanArgs& a, int B, cudaStream_t st) {
   switch (shape) {
-    case 208: return launch_one<T, 2, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
-    case 108: return launch_one<T, 1, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
-    case 104: return launch_one<T, 1, 4, PRECISE, ZOH, 0>(a, B, a.nch, st);
-    case 102: return launch_one<T, 1, 2, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 208: return launch_one<T, TD, 2, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 108: return launch_one<T, TD, 1, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 104: return launch_one<T, TD, 1, 4, PRECISE, ZOH, 0>(a, B, a.nch, st);
+    case 102: return launch_one<T, TD, 1, 2, PRECISE, ZOH, 0>(a, B, a.nch, st);
     default: return cudaErrorInvalidValue;
   }
 }
 
-template <typename T, bool PRECISE>
+template <typename T, typename TD, bool PRECISE>
 cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const float* h0, float* h_last,
                           float* chunk_ws, int num_sms, cudaStream_t st) {
   const bool zoh = c.disc_mode == 0;
   if (c.L == 1) {
     a.h0 = h0; a.h_last = h_last;
     dim3 grid((c.d_inner + BLOCK - 1) / BLOCK, c.B);
-    if (zoh) scan_step_kernel<T, PRECISE, true><<<grid, BLOCK, 0, st>>>(a);
-    else scan_step_kernel<T, PRECISE, false><<<grid, BLOCK, 0, st>>>(a);
+    if (zoh) scan_step_kernel<T, TD, PRECISE, true><<<grid, BLOCK, 0, st>>>(a);
+    else scan_step_kernel<T, TD, PRECISE, false><<<grid, BLOCK, 0, st>>>(a);
     count_launch();
     return cudaGetLastError();
   }
@@ -530,7 +531,7 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
   if (nch == 1) {
     a.Lc = c.L; a.L0 = c.L; a.nch = 1;
     const int shape = pick_thread_shape(c.B, c.d_inner, num_sms);
-    return zoh ? launch_shape<T, PRECISE, true>(shape, a, c.B, st) : launch_shape<T, PRECISE, false>(shape, a, c.B, st);
+    return zoh ? launch_shape<T, TD, PRECISE, true>(shape, a, c.B, st) : launch_shape<T, TD, PRECISE, false>(shape, a, c.B, st);
   }
   // chunked, two launches, 8 states per thread.  Launch A: chunk 0 in full from the caller's state, chunks
   // 1..n_end-1 state-only from zero; chain; launch B: chunks 1..nch-1 in full from their true initial states.
@@ -547,7 +548,7 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
   const int n_end = h_last ? nch : nch - 1;       // the last chunk's end state is only needed for h_last
   ScanArgs pa = a;
   pa.h_last = h_end; pa.sum_delta = sum_delta; pa.chunk_off = 0;
-  cudaError_t e = zoh ? launch_one<T, 1, 8, PRECISE, true, 2>(pa, c.B, n_end, st) : launch_one<T, 1, 8, PRECISE, false, 2>(pa, c.B, n_end, st);
+  cudaError_t e = zoh ? launch_one<T, TD, 1, 8, PRECISE, true, 2>(pa, c.B, n_end, st) : launch_one<T, TD, 1, 8, PRECISE, false, 2>(pa, c.B, n_end, st);
   if (e != cudaSuccess) return e;
   const long long n_thr = (long long)c.B * c.d_inner * NST;
   chain_chunk_states<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(A, h_end, sum_delta, h_in, h_last, c.B, c.d_inner, nch, n_end);
@@ -555,12 +556,12 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   a.h0 = h_in; a.h_last = nullptr; a.chunk_off = 1;
-  return zoh ? launch_one<T, 1, 8, PRECISE, true, 0>(a, c.B, nch - 1, st) : launch_one<T, 1, 8, PRECISE, false, 0>(a, c.B, nch - 1, st);
+  return zoh ? launch_one<T, TD, 1, 8, PRECISE, true, 0>(a, c.B, nch - 1, st) : launch_one<T, TD, 1, 8, PRECISE, false, 0>(a, c.B, nch - 1, st);
 }
 
 }  // namespace
 
-cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm,
+cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
                         void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st) {
   static int num_sms = 0;
@@ -572,8 +573,9 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const float* delta, 
     if (e != cudaSuccess) return e;
   }
   const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0};
-  return c.dtype == ROM_BF16 ? launch_scan_t<__nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
-                             : launch_scan_t<float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
+  if (c.dtype != ROM_BF16) return launch_scan_t<float, float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
+  return delta_fp32 ? launch_scan_t<__nv_bfloat16, float, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
+                    : launch_scan_t<__nv_bfloat16, __nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
 }
 
 }  // namespace rom

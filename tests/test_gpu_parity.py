@@ -165,7 +165,7 @@ def check_layer(s, recipe, with_D=True, gate_mode=0, disc_mode=0, flags=0, check
         assert_close(np64(g.tap("U", tdt, s.d_inner)), im["U"], tol, "U")
         assert_close(np64(g.tap("Bm", torch.float32, s.d_state)), im["Bm"], tol, "Bm")
         assert_close(np64(g.tap("Cm", torch.float32, s.d_state)), im["Cm"], tol, "Cm")
-        assert_close(np64(g.tap("Delta", torch.float32, s.d_inner)), im["Delta"], tol, "Delta")
+        assert_close(np64(g.tap("Delta", tdt, s.d_inner)), im["Delta"], tol, "Delta")
         rows = g.tap("row_of_assign", torch.int32, 1).view(-1)[::s.K].long()      # slot 0 row of each token
         assert_close(np64(g.tap("Ygp", tdt, s.d_inner)[rows]), im["Yg"], tol, "Yg")
     e = assert_close(np64(out), ref, tol, "out")
