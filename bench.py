@@ -36,8 +36,9 @@ UNIT = "tokens/s"
 # ncu capture, keyed by (stage, workload); None = not captured.  The summaries the figures come from
 # are the text files under profiles/.
 NCU_TRAFFIC_BYTES = {
-    # scan stage = first launch (395.6 MB) + second launch (612.0 MB) of the chunked scan; profiles/scan_long_ctx.md
-    ("scan", "long_ctx"): 1007.6e6,
+    # scan stage inside the layer (Delta in bf16) = first launch (269.0 MB) + second launch (478.5 MB) of the chunked
+    # scan; profiles/scan_long_ctx.md
+    ("scan", "long_ctx"): 747.5e6,
     # profiles/in_proj_long_ctx.md
     ("in_proj", "long_ctx"): 592.9e6,
 }
