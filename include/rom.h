@@ -38,7 +38,7 @@ typedef enum { ROM_F32 = 0, ROM_BF16 = 1 } rom_dtype;
 typedef enum {
   ROM_OK = 0,
   ROM_ERR_INVALID_ARG = -1,    /* NULL required pointer, bad size, misaligned pointer            */
-  ROM_ERR_UNSUPPORTED = -2,    /* a legal problem this build does not cover (e.g. d_state != 16)   */
+  ROM_ERR_UNSUPPORTED = -2,    /* a legal problem the library does not cover (e.g. d_state != 16)  */
   ROM_ERR_WORKSPACE = -3,      /* ws_bytes smaller than rom_workspace_size                        */
   ROM_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (launch, tensor-map encode)   */
   ROM_ERR_ARCH = -5,           /* the current device is not sm_100                                */
