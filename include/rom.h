@@ -220,13 +220,14 @@ ROM_API const char *rom_stage_name(int i);
 
 /* Locate a named intermediate of the last rom_layer_forward inside the workspace (host-only
  * arithmetic; for tests and debugging).  Names: "U" [T,D_e] dtype, "delta_r" [T,d_r] dtype,
- * "Bm","Cm" [T,D_s] f32, "Delta" [T,D_e] f32, "row_of_assign" [T*K] i32 (padded row of each
+ * "Bm","Cm" [T,D_s] f32, "Delta" [T,D_e] dtype, "row_of_assign" [T*K] i32 (padded row of each
  * assignment), "XZp" [rows,2*D_e] dtype, "Ygp" [rows,D_e] dtype, "pad_offsets" [E+1] i32.
  * Returns ROM_ERR_INVALID_ARG for an unknown name.                                                */
 ROM_API int rom_workspace_find(const rom_config *cfg, const char *name, size_t *offset, size_t *bytes);
 
-/* Read and clear the device status word of a workspace.  `host_code` (host out) receives ROM_OK or
- * ROM_ERR_DEVICE_TIMEOUT.  This call synchronises `stream`.                                       */
+/* Read and clear the device status word of a workspace.  `host_code` (host out) receives ROM_OK or the
+ * rom_status a kernel latched: ROM_ERR_DEVICE_TIMEOUT (a bounded wait expired) or ROM_ERR_INVALID_ARG
+ * (rom_ffn_moe_forward met an expert index out of range).  This call synchronises `stream`.       */
 ROM_API int rom_get_status(void *ws, void *stream, int32_t *host_code);
 
 /* Static string for a rom_status value.                                                           */
