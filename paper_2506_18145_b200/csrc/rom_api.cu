@@ -252,6 +252,10 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
 
   auto gemm = [&](const void* A_, int lda, const void* B_, int ldb, int n_experts, int64_t bstride, int M_max, int Nn, int Kd,
                   const int32_t* te, const int32_t* nmt, const Epilogue& ep) -> cudaError_t {
+    // a handful of rows against a long K (the x Proj of a single-token step): one 128-row tensor tile would be walked by a
+    // single CTA; the lane-split kernel spreads it over the GPU
+    if (!te && M_max <= 128 && Kd >= 1024 && Kd % 2048 == 0 && ep.mode == EPI_XPROJ)
+      return launch_gemm_skinny(c.dtype, A_, lda, B_, ldb, M_max, Nn, Kd, ep, st);
     if (tc) return launch_gemm_tc(A_, lda, B_, ldb, n_experts, M_max, Nn, Kd, te, nmt, ep, status, st);
     return launch_gemm_simt(c.dtype, A_, lda, B_, ldb, bstride, M_max, Nn, Kd, te, nmt, ep, st);
   };

@@ -8,6 +8,20 @@ namespace {
 
 constexpr int BM = 64, BN = 64, BK = 16;
 
+__device__ __forceinline__ void load_vec(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 q = __ldg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ void load_vec(const float* p, float (&v)[4]) {
+  const float4 q = __ldg(reinterpret_cast<const float4*>(p));
+  v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+}
+
 template <typename T>
 __device__ __forceinline__ void epi_store_scalar(const Epilogue& ep, int m, int n, float v) {
   switch (ep.mode) {
@@ -98,6 +112,58 @@ gemm_simt(const T* __restrict__ A, int lda, const T* __restrict__ Bw, int ldb, i
   }
 }
 
+// Few rows, long K (the x Proj of a single-token step): C[M,N] = A[M,Kd] * B[N,Kd]^T with the K dimension split over
+// all 256 threads of a block.  A block owns 2 rows x 4 columns, so a handful of rows still spreads over
+// (M/2) x (N/4) blocks and every thread has only Kd / (256 V) rounds of loads in flight behind one another
+// (V = 16 bytes of T; Kd % (256 V) == 0).  Partial sums: lanes by shuffles, then the 8 warps in warp order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+gemm_skinny(const T* __restrict__ A, int lda, const T* __restrict__ Bw, int ldb, int M, int N, int Kd, Epilogue ep) {
+  constexpr int V = 16 / sizeof(T);
+  __shared__ float part[8][8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n0 = blockIdx.x * 4;
+  const int r0 = blockIdx.y * 2;
+  const bool row1 = r0 + 1 < M;
+  float acc[2][4] = {};
+  for (int k = threadIdx.x * V; k < Kd; k += 256 * V) {
+    float a0[V], a1[V];
+    load_vec(A + (size_t)r0 * lda + k, a0);
+    if (row1) load_vec(A + (size_t)(r0 + 1) * lda + k, a1);
+    else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) a1[i] = 0.0f;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float w[V];
+      load_vec(Bw + (size_t)min(n0 + j, N - 1) * ldb + k, w);
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        acc[0][j] = fmaf(a0[i], w[i], acc[0][j]);
+        acc[1][j] = fmaf(a1[i], w[i], acc[1][j]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < 2; ++r)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float v = acc[r][j];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) part[warp][r * 4 + j] = v;
+    }
+  __syncthreads();
+  if (threadIdx.x < 8) {
+    const int r = threadIdx.x >> 2, j = threadIdx.x & 3;
+    float v = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) v += part[w][threadIdx.x];
+    if (r0 + r < M && n0 + j < N) epi_store_scalar<T>(ep, r0 + r, n0 + j, v);
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* Bw, int ldb, int64_t b_expert_stride,
@@ -110,6 +176,17 @@ cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* Bw, 
   else
     gemm_simt<float><<<grid, 256, 0, st>>>((const float*)A, lda, (const float*)Bw, ldb, b_expert_stride, M_max, N, Kd,
                                           tile_expert, num_m_tiles_dev, epi);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_skinny(int dtype, const void* A, int lda, const void* Bw, int ldb, int M, int N, int Kd,
+                               const Epilogue& epi, cudaStream_t st) {
+  dim3 grid((N + 3) / 4, (M + 1) / 2);
+  if (dtype == ROM_BF16)
+    gemm_skinny<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)A, lda, (const __nv_bfloat16*)Bw, ldb, M, N, Kd, epi);
+  else
+    gemm_skinny<float><<<grid, 256, 0, st>>>((const float*)A, lda, (const float*)Bw, ldb, M, N, Kd, epi);
   count_launch();
   return cudaGetLastError();
 }

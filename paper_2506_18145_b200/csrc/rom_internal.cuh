@@ -118,6 +118,11 @@ cudaError_t launch_gemm_simt(int dtype, const void* A, int lda, const void* Bw, 
                              int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
                              const Epilogue& epi, cudaStream_t st);
 
+// Ungrouped GEMM for a few rows and a long K (M <= 128, Kd a multiple of 2048 for bf16 / 1024 for fp32): K split over
+// the threads of a block.
+cudaError_t launch_gemm_skinny(int dtype, const void* A, int lda, const void* Bw, int ldb, int M, int N, int Kd,
+                               const Epilogue& epi, cudaStream_t st);
+
 cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int n_experts,
                            int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
                            const Epilogue& epi, int32_t* status, cudaStream_t st);

@@ -401,11 +401,12 @@ cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W
 
   const int n_wtiles = (c.E + NT8 - 1) / NT8;
   const int Epad8 = n_wtiles * NT8;
-  // warps per chunk: one per 8-expert tile, times a split of d_model (up to 4 ranges) that puts more loads in flight
-  int dsplit = 4;
+  // warps per chunk: one per 8-expert tile, times a split of d_model that puts more loads in flight: up to 4 ranges,
+  // up to 16 when there are too few chunks to fill the GPU (a handful of tokens: latency is all that matters)
+  const int blocks = (T + RT - 1) / RT;
+  int dsplit = blocks < 148 ? 16 : 4;
   while (dsplit > 1 && (n_wtiles * dsplit > 16 || c.d_model / 16 < 4 * dsplit)) dsplit >>= 1;
   const int threads = 32 * n_wtiles * dsplit;
-  const int blocks = (T + RT - 1) / RT;
   const bool bf = c.dtype == ROM_BF16;
   double* Wd = reinterpret_cast<double*>(ws + lay.wr_f64);
   const int nW = c.d_model * Epad8;

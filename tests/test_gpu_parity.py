@@ -338,6 +338,7 @@ def run_steps(s, n_steps, flags=0, routed_small=False):
     dict(B=5, L=12, E=8, K=1),
     dict(B=2, L=12, E=3, K=3, d_conv=3),
     dict(B=1, L=12, E=4, K=1, d_conv=2, dt_rank=32),
+    dict(B=5, L=12, E=4, K=1, d_inner=2048),                      # wide enough for the thread-split x Proj kernel
 ])
 @pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
 def test_layer_step_parity(kw, dtype, flags):
@@ -389,6 +390,7 @@ def test_layer_forward_host_matches_the_device_entry_point():
     dict(d_model=192, d_inner=320, dt_rank=48, E=5, K=2, B=2, L=257),      # widths that are multiples of 64 only
     dict(d_model=64, d_inner=64, dt_rank=16, E=2, K=1, B=1, L=700),        # the smallest widths
     dict(d_model=128, d_inner=192, dt_rank=16, E=64, K=8, B=1, L=300),     # the largest expert count and top-K
+    dict(d_model=128, d_inner=2048, dt_rank=16, E=4, K=2, B=1, L=99),      # few tokens, wide: thread-split x Proj kernel
 ])
 def test_layer_ragged_widths_and_limits(kw, dtype, flags):
     check_layer(small_shape(dtype=dtype, **kw), "unit", flags=flags)
