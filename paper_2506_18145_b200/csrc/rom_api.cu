@@ -289,15 +289,27 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
     // Per-expert x Proj / dt Proj under the same routing: U rows gathered into expert order (in the buffer the
     // scan fills later), two more grouped GEMMs over the existing row tiles, then the sum over the K slots.
     ROM_CUDA(launch_gather_rows_to(c, W + lay.U, W + lay.Ygp, De, W, lay, st));
-    Epilogue e_x{EPI_XPROJ, W + lay.delta_rp, R, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp), nullptr, R, N, nullptr, nullptr};
-    ROM_CUDA(gemm(W + lay.Ygp, De, w->W_x, De, c.E, (int64_t)(R + 2 * N) * De, (int)lay.rows_max, R + 2 * N, De, tile_expert, num_m_tiles, e_x));
-    ROM_STAGE_DONE();
-    Epilogue e_dt{EPI_F32, W + lay.Dpre, De, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
-    ROM_CUDA(gemm(W + lay.delta_rp, R, w->W_dt, R, c.E, (int64_t)De * R, (int)lay.rows_max, De, R, tile_expert, num_m_tiles, e_dt));
-    ROM_CUDA(launch_small_combine(c, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp),
-                                  reinterpret_cast<float*>(W + lay.Dpre), row_of_assign, w->b_dt, reinterpret_cast<float*>(W + lay.Bm),
-                                  reinterpret_cast<float*>(W + lay.Cm), W + lay.Delta, st));
-    ROM_STAGE_DONE();
+    if (tc && c.K == 1) {
+      // one expert per token on the tensor path: nothing to sum over slots, so the output ops put B, C and Delta
+      // (bias + softplus applied) straight at the token's row; only delta_r stays in expert order for the dt Proj
+      const int32_t* row_token = reinterpret_cast<const int32_t*>(W + lay.assign_of_row);
+      Epilogue e_x{EPI_XPROJ, W + lay.delta_rp, R, reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), nullptr, R, N, row_token, nullptr};
+      ROM_CUDA(gemm(W + lay.Ygp, De, w->W_x, De, c.E, (int64_t)(R + 2 * N) * De, (int)lay.rows_max, R + 2 * N, De, tile_expert, num_m_tiles, e_x));
+      ROM_STAGE_DONE();
+      Epilogue e_dt{EPI_SOFTPLUS_ROWS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0, row_token, nullptr};
+      ROM_CUDA(gemm(W + lay.delta_rp, R, w->W_dt, R, c.E, (int64_t)De * R, (int)lay.rows_max, De, R, tile_expert, num_m_tiles, e_dt));
+      ROM_STAGE_DONE();
+    } else {
+      Epilogue e_x{EPI_XPROJ, W + lay.delta_rp, R, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp), nullptr, R, N, nullptr, nullptr};
+      ROM_CUDA(gemm(W + lay.Ygp, De, w->W_x, De, c.E, (int64_t)(R + 2 * N) * De, (int)lay.rows_max, R + 2 * N, De, tile_expert, num_m_tiles, e_x));
+      ROM_STAGE_DONE();
+      Epilogue e_dt{EPI_F32, W + lay.Dpre, De, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
+      ROM_CUDA(gemm(W + lay.delta_rp, R, w->W_dt, R, c.E, (int64_t)De * R, (int)lay.rows_max, De, R, tile_expert, num_m_tiles, e_dt));
+      ROM_CUDA(launch_small_combine(c, reinterpret_cast<float*>(W + lay.Bp), reinterpret_cast<float*>(W + lay.Cp),
+                                    reinterpret_cast<float*>(W + lay.Dpre), row_of_assign, w->b_dt, reinterpret_cast<float*>(W + lay.Bm),
+                                    reinterpret_cast<float*>(W + lay.Cm), W + lay.Delta, st));
+      ROM_STAGE_DONE();
+    }
   }
   // S7 + S8 + S9: scan, gate, re-permute
   // K = 1: the gate row of a token is its Gate Proj row in expert order; K > 1: the summed rows from S4

@@ -42,7 +42,7 @@ constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 // Operand stages and epilogue staging per output op.  The softplus epilogue (dt Proj: only two K blocks per tile,
 // and the one GEMM here whose time is its fp32 output) gives up one operand stage for a 32 x 32 fp32 staging
 // square per epilogue warp, through which its stores become whole 128-byte row segments.
-__host__ __device__ constexpr bool f32_out(int mode) { return mode == EPI_SOFTPLUS || mode == EPI_F32; }
+__host__ __device__ constexpr bool f32_out(int mode) { return mode == EPI_SOFTPLUS || mode == EPI_F32 || mode == EPI_SOFTPLUS_ROWS; }
 __host__ __device__ constexpr int stages_of(int mode) { return f32_out(mode) ? 3 : MAX_STAGES; }
 __host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(mode) ? NUM_EPI_WARPS_C * 32 * 32 * 4 : 0; }
 __host__ __device__ constexpr int smem_bytes_of(int mode) {
@@ -133,7 +133,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
 // Bias of the 32 columns [n0, n0+32) (EPI_SOFTPLUS only), requested before the accumulator chunk is waited for.
 template <int MODE>
 __device__ __forceinline__ void load_bias(const Epilogue& ep, int n0, int N, float4 (&bq)[8]) {
-  if constexpr (MODE == EPI_SOFTPLUS) {
+  if constexpr (MODE == EPI_SOFTPLUS || MODE == EPI_SOFTPLUS_ROWS) {
 #pragma unroll
     for (int i = 0; i < 8; ++i)
       bq[i] = (ep.bias && n0 + 4 * i < N) ? __ldg(reinterpret_cast<const float4*>(ep.bias + n0) + i) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
@@ -142,9 +142,10 @@ __device__ __forceinline__ void load_bias(const Epilogue& ep, int n0, int N, flo
 
 // Fused output op on 32 consecutive accumulator columns [n0, n0+32) of row m (n0 % 32 == 0); columns at
 // or beyond N are skipped in groups of 8 (N % 8 == 0).
+// m: output row; m_tok (EPI_XPROJ with row_token only): row of the B / C parts, the token of this expert-order row.
 template <int MODE>
-__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0, int N, const uint32_t (&r)[32], float scale,
-                                            const float4 (&bq)[8]) {
+__device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, size_t m_tok, int n0, int N, const uint32_t (&r)[32],
+                                            float scale, const float4 (&bq)[8]) {
 #pragma unroll
   for (int j = 0; j < 32; j += 8) {
     const int n = n0 + j;
@@ -171,7 +172,7 @@ __device__ __forceinline__ void epi_store32(const Epilogue& ep, size_t m, int n0
       }
       *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + m * ld + n) = q;
     } else if (MODE == EPI_XPROJ) {
-      float* dst = (n < ep.R + ep.N) ? ep.Bm + m * ep.N + (n - ep.R) : ep.Cm + m * ep.N + (n - ep.R - ep.N);
+      float* dst = (n < ep.R + ep.N) ? ep.Bm + m_tok * ep.N + (n - ep.R) : ep.Cm + m_tok * ep.N + (n - ep.R - ep.N);
       *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
       *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
     } else {
@@ -222,8 +223,11 @@ __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, in
       __nv_bfloat162 h2 = __floats2bfloat162_rn(v1.x, v1.y), h3 = __floats2bfloat162_rn(v1.z, v1.w);
       q.x = *reinterpret_cast<uint32_t*>(&h0); q.y = *reinterpret_cast<uint32_t*>(&h1);
       q.z = *reinterpret_cast<uint32_t*>(&h2); q.w = *reinterpret_cast<uint32_t*>(&h3);
-      if (row0 + R < M_valid && n < N)
-        *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + (size_t)(row0 + R) * ep.ldc + n) = q;
+      if (row0 + R < M_valid && n < N) {
+        // per-expert dt Proj at top-1: the row goes to its token's position (padding rows are skipped)
+        const int orow = MODE == EPI_SOFTPLUS_ROWS ? __ldg(ep.row_token + row0 + R) : row0 + R;
+        if (orow >= 0) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + (size_t)orow * ep.ldc + n) = q;
+      }
     }
   }
   __syncwarp();
@@ -360,6 +364,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool row_ok = row < M_valid;
       size_t out_row = (size_t)row;
       float scale = 1.0f;
+      size_t tok_row = (size_t)row;
       if ((MODE == EPI_OUTPROJ || (MODE == EPI_INPROJ && ep.row_token != nullptr)) && row_ok) {
         const int tok = __ldg(ep.row_token + row);      // rows are written at their token's position
         row_ok = tok >= 0;
@@ -367,6 +372,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           out_row = (size_t)tok;
           if (MODE == EPI_OUTPROJ) scale = __ldg(ep.row_scale + tok);
         }
+      }
+      if (MODE == EPI_XPROJ && ep.row_token != nullptr && row_ok) {
+        // per-expert x Proj at top-1: delta_r stays in expert order (it feeds the grouped dt Proj), B and C go to the token's row
+        const int tok = __ldg(ep.row_token + row);
+        row_ok = tok >= 0;
+        tok_row = row_ok ? (size_t)tok : 0;
       }
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * MAX_BLOCK_N;
       const int n_base = n_tile * block_n;
@@ -405,14 +416,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         tmem_ld_wait(ra);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
         if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
-        else if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, ra, scale, bq);
+        else if (row_ok) epi_store32<MODE>(ep, out_row, tok_row, n_base + ch * 32, N, ra, scale, bq);
         ch += 2;
         if (ch >= n_chunks) break;
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);
         tmem_ld_wait(rb);
         if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
         if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
-        else if (row_ok) epi_store32<MODE>(ep, out_row, n_base + ch * 32, N, rb, scale, bq);
+        else if (row_ok) epi_store32<MODE>(ep, out_row, tok_row, n_base + ch * 32, N, rb, scale, bq);
         ch += 2;
       }
       tc_fence_before();
@@ -489,6 +500,7 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
               : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : epi.mode == EPI_OUTPROJ ? gemm_tc_kernel<EPI_OUTPROJ>
               : epi.mode == EPI_F32 ? gemm_tc_kernel<EPI_F32> : epi.mode == EPI_SWIGLU ? gemm_tc_kernel<EPI_SWIGLU>
+              : epi.mode == EPI_SOFTPLUS_ROWS ? gemm_tc_kernel<EPI_SOFTPLUS_ROWS>
               : gemm_tc_kernel<EPI_SOFTPLUS>;
   const int smem_bytes = smem_bytes_of(epi.mode);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);

@@ -69,8 +69,9 @@ enum EpiMode : int {
   EPI_OUTPROJ = 4,    // top-1 combine fused: C[row_token[m], n] = row_scale[row_token[m]] * acc; rows with
                       // row_token[m] < 0 (segment padding) are skipped   (dtype; tensor path only)
   EPI_F32 = 5,        // C[m, n] = acc                          (fp32)
-  EPI_SWIGLU = 6      // C[m, j] = SiLU(acc[m, j]) * acc[m, N + j], j < N: B holds, per expert, N "gate" rows then N "up"
+  EPI_SWIGLU = 6,     // C[m, j] = SiLU(acc[m, j]) * acc[m, N + j], j < N: B holds, per expert, N "gate" rows then N "up"
                       // rows; N % 128 == 0   (dtype; tensor path only)
+  EPI_SOFTPLUS_ROWS = 7  // EPI_SOFTPLUS with row m written at row row_token[m] (skipped when negative)   (tensor path only)
 };
 struct Epilogue {
   int mode;
