@@ -507,7 +507,6 @@ int pick_thread_shape(int B, int De, int num_sms) {
 template <typename T, typename TD, bool PRECISE, bool ZOH>
 cudaError_t launch_shape(int shape, const ScanArgs& a, int B, cudaStream_t st) {
   switch (shape) {
-    case 208: return launch_one<T, TD, 2, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
     case 108: return launch_one<T, TD, 1, 8, PRECISE, ZOH, 0>(a, B, a.nch, st);
     case 104: return launch_one<T, TD, 1, 4, PRECISE, ZOH, 0>(a, B, a.nch, st);
     case 102: return launch_one<T, TD, 1, 2, PRECISE, ZOH, 0>(a, B, a.nch, st);
