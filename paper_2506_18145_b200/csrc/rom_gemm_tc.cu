@@ -43,10 +43,16 @@ constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 // and the one GEMM here whose time is its fp32 output) gives up one operand stage for a 32 x 32 fp32 staging
 // square per epilogue warp, through which its stores become whole 128-byte row segments.
 __host__ __device__ constexpr bool f32_out(int mode) { return mode == EPI_SOFTPLUS || mode == EPI_F32 || mode == EPI_SOFTPLUS_ROWS; }
-__host__ __device__ constexpr int stages_of(int mode) { return f32_out(mode) ? 3 : MAX_STAGES; }
+// The x Proj (a narrow B tile, one wave of row tiles, time set by how many bytes of A are in flight) runs six
+// smaller stages: its B tile is at most XPROJ_BLOCK_N rows.
+constexpr int XPROJ_BLOCK_N = 160;
+__host__ __device__ constexpr int stage_bytes_of(int mode) {
+  return mode == EPI_XPROJ ? A_STAGE_BYTES + XPROJ_BLOCK_N * BLOCK_K * 2 : STAGE_BYTES;
+}
+__host__ __device__ constexpr int stages_of(int mode) { return f32_out(mode) ? 3 : mode == EPI_XPROJ ? 6 : MAX_STAGES; }
 __host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(mode) ? NUM_EPI_WARPS_C * 32 * 32 * 4 : 0; }
 __host__ __device__ constexpr int smem_bytes_of(int mode) {
-  return stages_of(mode) * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
+  return stages_of(mode) * stage_bytes_of(mode) + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
 }
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait polls before a wait gives up (a few seconds)
 
@@ -240,18 +246,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ num_m_tiles_dev,
                Epilogue ep, int32_t* __restrict__ status) {
   constexpr int STAGES = stages_of(MODE);
+  constexpr int SB = stage_bytes_of(MODE);          // bytes per operand stage (multiple of 1024)
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;               // 128B-swizzled tiles need 1024-byte alignment
   unsigned char* smem = smem_raw + (base - raw);
-  const uint32_t bars = base + STAGES * STAGE_BYTES;          // barrier block (8-byte aligned)
+  const uint32_t bars = base + STAGES * SB;                   // barrier block (8-byte aligned)
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + ACC_STAGES + a); };
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 2 * ACC_STAGES));
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + STAGES * SB + 8 * (2 * STAGES + 2 * ACC_STAGES));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
-  float* out_stage = reinterpret_cast<float*>(smem + STAGES * STAGE_BYTES + 256);        // [8 warps][32][32] (softplus only)
+  float* out_stage = reinterpret_cast<float*>(smem + STAGES * SB + 256);        // [8 warps][32][32] (softplus only)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -293,7 +300,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), stage_tx);
-          const uint32_t sa = base + stage * STAGE_BYTES;
+          const uint32_t sa = base + stage * SB;
           tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BLOCK_K, m_tile * BLOCK_M);
           tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row);
           if (MODE == EPI_SWIGLU)     // second half of the B tile: the up rows of the same 128 hidden units (box = 128 rows)
@@ -329,7 +336,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = base + stage * STAGE_BYTES;
+          const uint32_t sa = base + stage * SB;
           const uint64_t adesc = make_smem_desc(sa);
           const uint64_t bdesc = make_smem_desc(sa + A_STAGE_BYTES);
 #pragma unroll
@@ -483,6 +490,7 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   const bool swiglu = epi.mode == EPI_SWIGLU;      // N output columns from 2N rows of B per expert, loaded as two boxes of 128 rows
   if (swiglu && (N % 128 != 0 || MAX_BLOCK_N != 256)) return cudaErrorInvalidValue;
   int block_n = (swiglu || N >= MAX_BLOCK_N) ? MAX_BLOCK_N : (N + 31) / 32 * 32;
+  if (epi.mode == EPI_XPROJ && block_n > XPROJ_BLOCK_N) block_n = XPROJ_BLOCK_N;
   CUtensorMap ta, tb;
   if (!make_tmap(&ta, A, (uint64_t)M_max, (uint64_t)Kd, (uint64_t)lda, BLOCK_M)) return cudaErrorInvalidValue;
   if (!make_tmap(&tb, Bw, (uint64_t)n_experts * (swiglu ? 2 * N : N), (uint64_t)Kd, (uint64_t)ldb, swiglu ? 128u : (uint32_t)block_n))
