@@ -18,7 +18,7 @@
 // the MMAs of tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches an error code in
 // the status word, drains its own copies with a bounded wait, frees its TMEM and returns.
 //
-// No cluster multicast is used anywhere in this file.
+// Every TMA load here is a plain single-CTA load (no thread-block clusters).
 #include <cuda.h>
 
 #include "rom_internal.cuh"
