@@ -39,6 +39,10 @@ constexpr int ACC_STAGES = 2;
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_EPI_WARPS = NUM_EPI_WARPS_C;
 constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
+// The dt Proj (softplus output ops) has two K blocks per tile and about ten instructions plus two special-function
+// operations per output element: its time is its epilogue's, so it runs sixteen epilogue warps instead of eight.
+__host__ __device__ constexpr int epi_warps_of(int mode) { return (mode == EPI_SOFTPLUS || mode == EPI_SOFTPLUS_ROWS) ? 16 : NUM_EPI_WARPS_C; }
+__host__ __device__ constexpr int threads_of(int mode) { return 64 + 32 * epi_warps_of(mode); }
 // Operand stages and epilogue staging per output op.  The softplus epilogue (dt Proj: only two K blocks per tile,
 // and the one GEMM here whose time is its fp32 output) gives up one operand stage for a 32 x 32 fp32 staging
 // square per epilogue warp, through which its stores become whole 128-byte row segments.
@@ -50,7 +54,7 @@ __host__ __device__ constexpr int stage_bytes_of(int mode) {
   return mode == EPI_XPROJ ? A_STAGE_BYTES + XPROJ_BLOCK_N * BLOCK_K * 2 : STAGE_BYTES;
 }
 __host__ __device__ constexpr int stages_of(int mode) { return f32_out(mode) ? 3 : mode == EPI_XPROJ ? 6 : MAX_STAGES; }
-__host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(mode) ? NUM_EPI_WARPS_C * 32 * 32 * 4 : 0; }
+__host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(mode) ? epi_warps_of(mode) * 32 * 32 * 4 : 0; }
 __host__ __device__ constexpr int smem_bytes_of(int mode) {
   return stages_of(mode) * stage_bytes_of(mode) + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
 }
@@ -240,7 +244,7 @@ __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, in
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(threads_of(MODE), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M_max, int N, int Kd, int block_n, uint32_t idesc,
                const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ num_m_tiles_dev,
@@ -273,7 +277,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), NUM_EPI_WARPS); }
+    for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), epi_warps_of(MODE)); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -359,7 +363,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter+32) belong to this warp
-    const int half = (warp - 2) >> 2;             // which of the two warps of the quarter: takes chunks half, half+2, ...
+    constexpr int EWQ = epi_warps_of(MODE) / 4;   // warps per lane quarter
+    const int half = (warp - 2) >> 2;             // which of the EWQ warps of the quarter: takes chunks half, half+EWQ, ...
     const int n_chunks = block_n >> 5;
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
@@ -415,23 +420,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
         }
       }
-      int ch = MODE == EPI_SWIGLU ? n_chunks : half;
+      if constexpr (EWQ == 4) {
+        // sixteen warps: at most two chunks each, one register buffer (the register file has no room for two)
+        for (int c = half; c < n_chunks; c += EWQ) {
+          tmem_ld32_issue(taddr + c * 32, ra);
+          load_bias<MODE>(ep, n_base + c * 32, N, bq);
+          tmem_ld_wait(ra);
+          epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + c * 32, N, ra, bq, lane);
+        }
+      }
+      int ch = (MODE == EPI_SWIGLU || EWQ == 4) ? n_chunks : half;
       if (ch < n_chunks) tmem_ld32_issue(taddr + ch * 32, ra);
       // two register buffers: while one chunk is processed the next chunk's tensor-memory load is in flight
       while (ch < n_chunks) {
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);     // in flight together with the tensor-memory load
         tmem_ld_wait(ra);
-        if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, rb);
+        if (ch + EWQ < n_chunks) tmem_ld32_issue(taddr + (ch + EWQ) * 32, rb);
         if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
         else if (row_ok) epi_store32<MODE>(ep, out_row, tok_row, n_base + ch * 32, N, ra, scale, bq);
-        ch += 2;
+        ch += EWQ;
         if (ch >= n_chunks) break;
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);
         tmem_ld_wait(rb);
-        if (ch + 2 < n_chunks) tmem_ld32_issue(taddr + (ch + 2) * 32, ra);
+        if (ch + EWQ < n_chunks) tmem_ld32_issue(taddr + (ch + EWQ) * 32, ra);
         if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
         else if (row_ok) epi_store32<MODE>(ep, out_row, tok_row, n_base + ch * 32, N, rb, scale, bq);
-        ch += 2;
+        ch += EWQ;
       }
       tc_fence_before();
       __syncwarp();
@@ -516,7 +530,7 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   const int n_tiles = swiglu ? N / 128 : (N + block_n - 1) / block_n;
   const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
   const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
-  kern<<<grid, NUM_THREADS, smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
+  kern<<<grid, threads_of(epi.mode), smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
   count_launch();
   return cudaGetLastError();
 }
