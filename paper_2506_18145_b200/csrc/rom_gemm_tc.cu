@@ -204,8 +204,8 @@ __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, in
       o = make_float4(__uint_as_float(r[4 * c]), __uint_as_float(r[4 * c + 1]), __uint_as_float(r[4 * c + 2]), __uint_as_float(r[4 * c + 3]));
     } else {
       const float4 b = bq[c];
-      o = make_float4(softplus_fast(__uint_as_float(r[4 * c]) + b.x), softplus_fast(__uint_as_float(r[4 * c + 1]) + b.y),
-                      softplus_fast(__uint_as_float(r[4 * c + 2]) + b.z), softplus_fast(__uint_as_float(r[4 * c + 3]) + b.w));
+      o = make_float4(softplus_bf16(__uint_as_float(r[4 * c]) + b.x), softplus_bf16(__uint_as_float(r[4 * c + 1]) + b.y),
+                      softplus_bf16(__uint_as_float(r[4 * c + 2]) + b.z), softplus_bf16(__uint_as_float(r[4 * c + 3]) + b.w));
     }
     *reinterpret_cast<float4*>(sw + lane * 32 + ((c ^ (lane & 7)) << 2)) = o;
   }
@@ -241,6 +241,41 @@ __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, in
     }
   }
   __syncwarp();
+}
+
+// Softplus output op for sixteen epilogue warps: a warp owns two adjacent 32-column chunks of its 32 rows.  Every lane
+// activates and rounds its row of a chunk to bf16 and stages it (swizzled 16-byte pieces, 128 bytes per row for the two
+// chunks); after the second chunk the warp writes whole 128-byte row segments, four rows per store instruction.
+// stage: 32 rows x 8 pieces of 16 bytes.  piece0: first piece of this chunk (0 or 4).
+__device__ __forceinline__ void softplus_stage_bf16(uint4* stage, int piece0, const uint32_t (&r)[32], const float4 (&bq)[8], int lane) {
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float4 b0 = bq[2 * j], b1 = bq[2 * j + 1];
+    uint4 q;
+    __nv_bfloat162 h0 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j]) + b0.x), softplus_bf16(__uint_as_float(r[8 * j + 1]) + b0.y));
+    __nv_bfloat162 h1 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j + 2]) + b0.z), softplus_bf16(__uint_as_float(r[8 * j + 3]) + b0.w));
+    __nv_bfloat162 h2 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j + 4]) + b1.x), softplus_bf16(__uint_as_float(r[8 * j + 5]) + b1.y));
+    __nv_bfloat162 h3 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j + 6]) + b1.z), softplus_bf16(__uint_as_float(r[8 * j + 7]) + b1.w));
+    q.x = *reinterpret_cast<uint32_t*>(&h0); q.y = *reinterpret_cast<uint32_t*>(&h1);
+    q.z = *reinterpret_cast<uint32_t*>(&h2); q.w = *reinterpret_cast<uint32_t*>(&h3);
+    stage[lane * 8 + ((piece0 + j) ^ (lane & 7))] = q;
+  }
+}
+// n0: column of piece 0; pieces at or beyond n_pieces (0, 4 or 8 valid) or beyond N are not written.
+template <int MODE>
+__device__ __forceinline__ void softplus_flush_bf16(const Epilogue& ep, const uint4* stage, int row0, int M_valid, int n0, int N,
+                                                    int n_pieces, int lane) {
+  const int p = lane & 7;
+  const int n = n0 + 8 * p;
+#pragma unroll
+  for (int r4 = 0; r4 < 8; ++r4) {
+    const int R = r4 * 4 + (lane >> 3);
+    const uint4 q = stage[R * 8 + (p ^ (R & 7))];
+    if (row0 + R < M_valid && p < n_pieces && n < N) {
+      const int orow = MODE == EPI_SOFTPLUS_ROWS ? __ldg(ep.row_token + row0 + R) : row0 + R;
+      if (orow >= 0) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + (size_t)orow * ep.ldc + n) = q;
+    }
+  }
 }
 
 template <int MODE>
@@ -422,11 +457,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
       if constexpr (EWQ == 4) {
         // sixteen warps: at most two chunks each, one register buffer (the register file has no room for two)
-        for (int c = half; c < n_chunks; c += EWQ) {
-          tmem_ld32_issue(taddr + c * 32, ra);
-          load_bias<MODE>(ep, n_base + c * 32, N, bq);
+        uint4* stage = reinterpret_cast<uint4*>(out_stage + (warp - 2) * 1024);
+        const int c0 = 2 * half;                       // this warp's chunks: c0 and c0 + 1
+        int n_pieces = 0;
+        for (int cc = 0; cc < 2 && c0 + cc < n_chunks; ++cc) {
+          tmem_ld32_issue(taddr + (c0 + cc) * 32, ra);
+          load_bias<MODE>(ep, n_base + (c0 + cc) * 32, N, bq);
           tmem_ld_wait(ra);
-          epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + c * 32, N, ra, bq, lane);
+          softplus_stage_bf16(stage, 4 * cc, ra, bq, lane);
+          n_pieces += 4;
+        }
+        if (n_pieces > 0) {
+          __syncwarp();
+          softplus_flush_bf16<MODE>(ep, stage, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + c0 * 32, N, n_pieces, lane);
+          __syncwarp();
         }
       }
       int ch = (MODE == EPI_SWIGLU || EWQ == 4) ? n_chunks : half;
