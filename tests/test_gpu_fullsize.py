@@ -4,9 +4,11 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import rom_oracle as O
+from paper_2506_18145_b200 import binding as rb
 from paper_2506_18145_b200 import synth
 
-from rom_testlib import TOL, GpuLayer, assert_close, np64, oracle_layer
+from rom_testlib import TOL, GpuLayer, assert_close, gpu_route, np64, oracle_layer
 
 pytestmark = pytest.mark.gpu
 
@@ -28,3 +30,50 @@ def test_layer_full_size(name):
     np.testing.assert_allclose(gates, im["gate"], rtol=2e-6)
     assert_close(Yg, im["Yg"], TOL["bf16"], "Yg")
     assert_close(out, ref, TOL["bf16"], "out")
+
+
+def test_ffn_moe_full_size_sampled_tokens():
+    """FFN-MoE with shared routing at the benchmark shape (`bench.py --stage ffn`: long_ctx widths, d_ff = 4 d_model):
+    the experts are per-token functions, so the oracle is evaluated on a sample of 384 tokens (every 43rd)."""
+    s = synth.CONFIGS["long_ctx"]
+    d_ff = 4 * s.d_model
+    p = synth.make_inputs(s.replace(d_inner=64, dt_rank=16))
+    g = torch.Generator().manual_seed(s.seed_base + 900)
+    W_gu = (torch.randn((s.E, 2 * d_ff, s.d_model), generator=g) * 0.02).to(torch.bfloat16)
+    W_down = (torch.randn((s.E, s.d_model, d_ff), generator=g) * 0.02).to(torch.bfloat16)
+    r = gpu_route(s, p)
+    cfg = rb.config_from_shape(s)
+    idx = torch.from_numpy(r["idx"]).cuda(); gates = torch.from_numpy(r["gates"]).cuda()
+    ws = torch.empty(rb.ffn_moe_workspace_size(cfg, d_ff), dtype=torch.uint8, device="cuda")
+    out = torch.empty((s.B, s.L, s.d_model), dtype=torch.bfloat16, device="cuda")
+    rb.rom_ffn_moe_forward(cfg, d_ff, W_gu.cuda(), W_down.cuda(), p["x"].cuda(), idx, gates, out, ws)
+    torch.cuda.synchronize()
+    assert rb.rom_get_status(ws) == 0
+    sample = np.arange(0, s.T, 43)[:384]
+    x = np64(p["x"]).reshape(s.T, s.d_model)[sample]
+    ref = O.ffn_moe_shared_routing(x, np64(W_gu), np64(W_down), r["idx"][sample], r["gates"][sample].astype(np.float64))
+    assert_close(np64(out).reshape(s.T, s.d_model)[sample], ref, TOL["bf16"], "ffn out (sampled tokens)")
+
+
+def test_layer_step_full_size():
+    """Single-token step at the benchmark shape (`bench.py --stage step`: 64 sequences, long_ctx widths): three steps
+    against the oracle's step with states carried on both sides."""
+    s = synth.CONFIGS["long_ctx"].replace(B=64, L=3)
+    p = synth.make_inputs(s, recipe="unit")
+    cfg = rb.config_from_shape(s.replace(L=1))
+    dev = {k: (None if v is None else v.cuda().contiguous()) for k, v in p.items()}
+    weights = rb.make_weights(dev)
+    ws = rb.alloc_workspace(cfg, "cuda")
+    conv_state = torch.zeros((s.B, s.d_conv - 1, s.d_inner), dtype=torch.float32, device="cuda")
+    ssm_state = torch.zeros((s.B, s.d_inner, s.d_state), dtype=torch.float32, device="cuda")
+    out = torch.empty((s.B, s.d_model), dtype=torch.bfloat16, device="cuda")
+    o_conv = np.zeros((s.B, s.d_conv - 1, s.d_inner)); o_h = np.zeros((s.B, s.d_inner, s.d_state))
+    wn = [np64(p[k]) for k in ("W_r", "b_r", "W_inz", "w_conv", "b_conv", "W_x", "W_dt", "b_dt", "A", "D", "W_out")]
+    for t in range(s.L):
+        rb.rom_layer_step(cfg, weights, dev["x"][:, t].contiguous(), conv_state, ssm_state, out, None, None, ws)
+        torch.cuda.synchronize()
+        assert rb.rom_get_status(ws) == 0
+        ref, o_conv, o_h = O.rom_layer_step(np64(p["x"][:, t]), o_conv, o_h, *wn, K=s.K, dt_rank=s.dt_rank)
+        assert_close(np64(out), ref, TOL["bf16"], f"step {t} out")
+    assert_close(np64(ssm_state), o_h, TOL["bf16"], "state-space state")
+
