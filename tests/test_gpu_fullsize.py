@@ -77,3 +77,36 @@ def test_layer_step_full_size():
         assert_close(np64(out), ref, TOL["bf16"], f"step {t} out")
     assert_close(np64(ssm_state), o_h, TOL["bf16"], "state-space state")
 
+
+def test_layer_full_size_per_expert_small_projections():
+    """The per-expert x Proj / dt Proj mode (`bench.py --small-proj routed`) at the benchmark workload."""
+    s = synth.CONFIGS["long_ctx"]
+    p = synth.make_inputs(s, routed_small=True)
+    g = GpuLayer(s, p)
+    out = np64(g.forward())
+    idx = g.idx.cpu().numpy()
+    del g
+    torch.cuda.empty_cache()
+    ref, im = oracle_layer(s, p)
+    np.testing.assert_array_equal(idx, im["idx"])
+    assert_close(out, ref, TOL["bf16"], "out")
+
+
+@pytest.mark.parametrize("name", ["long_ctx", "zipf"])
+def test_route_balance_full_size(name):
+    """Load-balance statistic of the router (Appendix A.3) at benchmark sizes."""
+    s = synth.CONFIGS[name]
+    p = synth.make_inputs(s.replace(d_inner=64, dt_rank=16))
+    cfg = rb.config_from_shape(s)
+    ws = rb.alloc_workspace(cfg)
+    F = torch.empty(s.E, dtype=torch.float32, device="cuda"); Pb = torch.empty_like(F)
+    loss = torch.empty(1, dtype=torch.float32, device="cuda")
+    b_r = None if p["b_r"] is None else p["b_r"].cuda()
+    rb.rom_route_balance(cfg, p["x"].cuda(), p["W_r"].cuda(), b_r, 1e-3, F, Pb, loss, ws)
+    torch.cuda.synchronize()
+    idx, gate, P, logit = O.route(np64(p["x"]).reshape(s.T, s.d_model), np64(p["W_r"]), np64(p["b_r"]), s.K)
+    want, Fr = O.load_balance_loss(P, idx, alpha=1e-3)
+    np.testing.assert_allclose(F.cpu().numpy(), Fr, rtol=1e-6)
+    np.testing.assert_allclose(Pb.cpu().numpy(), P.mean(axis=0), rtol=2e-6)
+    np.testing.assert_allclose(float(loss.item()), want, rtol=2e-6)
+
