@@ -24,3 +24,11 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library_is_built():
+    """Build the CUDA library in-tree if it is missing or older than its sources (a no-op otherwise), so the
+    tests always run against the current code.  There is no fallback: a build failure fails the session."""
+    from paper_2506_18145_b200 import build as rbuild
+    rbuild.build()
