@@ -181,7 +181,7 @@ def run_stage(args, s):
         q = synth.make_scan_inputs(s.B, s.L, s.d_inner, s.d_state, s.dtype, s.seed_base + 500)
         d = {k: (None if v is None else v.to(dev)) for k, v in q.items()}
         y = torch.empty_like(d["u"])
-        ws = rb.alloc_workspace(cfg, dev)
+        ws = torch.empty(max(rb.scan_workspace_size(cfg), 16), dtype=torch.uint8, device=dev)
         call = lambda: rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], None, y, None, ws)
         esz = 2 if s.dtype == "bf16" else 4
         nbytes = s.T * (4 * s.d_inner * esz + 8 * s.d_state)        # u, Delta, z, y at storage width; B, C fp32

@@ -83,8 +83,14 @@ typedef struct {                /* all read-only device pointers                
   const void  *W_out;           /* [E, d_model, d_inner]     dtype  W_out,i^T                      */
 } rom_weights;
 
-/* Bytes of workspace rom_layer_forward / rom_route / rom_scan need for this config (host out).   */
+/* Bytes of workspace rom_layer_forward / rom_route / rom_route_balance / rom_layer_step need for this
+ * config (host out).                                                                              */
 ROM_API int rom_workspace_size(const rom_config *cfg, size_t *bytes);
+
+/* Bytes of workspace with which rom_scan cuts a long sequence into chunks that run in parallel (host out;
+ * a few MB: two states and one sum of Delta per chunk, sequence and channel).  0 when batch x channels
+ * already fill the GPU and the sequence is scanned in one pass.  Uses cfg->B, L, d_inner, d_state, dtype. */
+ROM_API int rom_scan_workspace_size(const rom_config *cfg, size_t *bytes);
 
 /* Router + top-K + dropless permutation (Section 4.2 routing equation; Section 5.1: no capacity
  * factor, no token dropping).
@@ -144,6 +150,8 @@ ROM_API int rom_route_noalloc(const rom_config *cfg, const void *x, const void *
  *   u, z, y : [B, L, d_inner] dtype;  delta : [B, L, d_inner] fp32;  A : [d_inner, d_state] fp32;
  *   Bm, Cm : [B, L, d_state] fp32;  D : [d_inner] or NULL;  z NULL = no gate;
  *   h0 : [B, d_inner, d_state] fp32 or NULL (zeros);  h_last : same shape or NULL (not produced).
+ *   ws : NULL (one pass per sequence, whatever its length) or at least rom_scan_workspace_size(cfg) bytes
+ *        (a larger buffer, e.g. the layer's workspace, is accepted; only its head is used).
  * Uses cfg->B, L, d_inner, d_state, dtype, disc_mode.                                             */
 ROM_API int rom_scan(const rom_config *cfg, const void *u, const float *delta, const float *A,
              const float *Bm, const float *Cm, const float *D, const void *z, const float *h0,

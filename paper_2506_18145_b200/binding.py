@@ -22,7 +22,8 @@ ROM_OK = 0
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
            "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance",
-           "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step", "rom_layer_forward_host")
+           "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step", "rom_layer_forward_host",
+           "rom_scan_workspace_size")
 
 
 class RomConfig(ctypes.Structure):
@@ -56,6 +57,7 @@ def lib() -> ctypes.CDLL:
         vp, i32p, szp = ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(ctypes.c_size_t)
         cfgp = ctypes.POINTER(RomConfig)
         L.rom_workspace_size.argtypes = [cfgp, szp]
+        L.rom_scan_workspace_size.argtypes = [cfgp, szp]
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
         L.rom_route_noalloc.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
         L.rom_route_balance.argtypes = [cfgp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -117,6 +119,14 @@ def workspace_size(cfg: RomConfig) -> int:
     rc = lib().rom_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
     if rc != ROM_OK:
         raise RomError(rc, "rom_workspace_size")
+    return int(n.value)
+
+
+def scan_workspace_size(cfg: RomConfig) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().rom_scan_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_scan_workspace_size")
     return int(n.value)
 
 

@@ -123,6 +123,14 @@ int rom_workspace_size(const rom_config* cfg, size_t* bytes) {
   return ROM_OK;
 }
 
+int rom_scan_workspace_size(const rom_config* cfg, size_t* bytes) {
+  if (!bytes) return ROM_ERR_INVALID_ARG;
+  const int rc = check_config(cfg, 2);
+  if (rc != ROM_OK) return rc;
+  *bytes = align_up(sizeof(float) * scan_ws_floats(cfg->B, cfg->d_inner, cfg->L), 256);
+  return ROM_OK;
+}
+
 int rom_workspace_find(const rom_config* cfg, const char* name, size_t* offset, size_t* bytes) {
   if (!cfg || !name || !offset || !bytes) return ROM_ERR_INVALID_ARG;
   const WsLayout l = make_layout(*cfg);
@@ -183,16 +191,12 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
   if ((rc = check_device()) != ROM_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   LaunchCounter::count = 0;
-  // with a workspace of rom_workspace_size bytes a long sequence is scanned in parallel chunks; without one, in one pass
+  // with a workspace of rom_scan_workspace_size bytes a long sequence is scanned in parallel chunks; without one, in one pass
   float* chunk_ws = nullptr;
   if (ws != nullptr) {
     if (!aligned16(ws)) return ROM_ERR_INVALID_ARG;
-    rom_config full = *cfg;
-    if (full.E < 1) full.E = 1;
-    if (full.K < 1) full.K = 1;
-    const WsLayout lay = make_layout(full);
-    if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
-    chunk_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + lay.scan_ws);
+    if (ws_bytes < sizeof(float) * scan_ws_floats(cfg->B, cfg->d_inner, cfg->L)) return ROM_ERR_WORKSPACE;
+    chunk_ws = static_cast<float*>(ws);
   }
   ROM_CUDA(launch_scan(*cfg, u, delta, true, A, Bm, Cm, D, z, cfg->d_inner, nullptr, h0, y, h_last, nullptr, 1, chunk_ws, false, st));
   return ROM_OK;

@@ -13,23 +13,72 @@ from rom_testlib import TOL, GpuLayer, assert_close, gpu_route, np64, oracle_lay
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name", ["long_ctx", "zipf", "short_seqs"])
-def test_layer_full_size(name):
-    s = synth.CONFIGS[name]
-    p = synth.make_inputs(s)
+def _layer_full_size(s, p):
+    """Forward on the GPU and on the oracle; routing bit-exact; every tap the small-shape tests compare (U, B, C, Delta,
+    gated scan output) and the layer output within the bf16 tolerance."""
     g = GpuLayer(s, p)
     out = np64(g.forward())
     idx = g.idx.cpu().numpy(); counts = g.counts.cpu().numpy(); gates = g.gates.cpu().numpy()
+    tdt = synth.torch_dtype(s)
     Yg_rows = g.tap("row_of_assign", torch.int32, 1).view(-1)[::s.K].long()
-    Yg = np64(g.tap("Ygp", synth.torch_dtype(s), s.d_inner)[Yg_rows])
+    taps = {"Yg": np64(g.tap("Ygp", tdt, s.d_inner)[Yg_rows]),
+            "U": np64(g.tap("U", tdt, s.d_inner)),
+            "Bm": np64(g.tap("Bm", torch.float32, s.d_state)),
+            "Cm": np64(g.tap("Cm", torch.float32, s.d_state)),
+            "Delta": np64(g.tap("Delta", tdt, s.d_inner))}
     del g
     torch.cuda.empty_cache()
     ref, im = oracle_layer(s, p)
     np.testing.assert_array_equal(idx, im["idx"])
     np.testing.assert_array_equal(counts, im["counts"])
     np.testing.assert_allclose(gates, im["gate"], rtol=2e-6)
-    assert_close(Yg, im["Yg"], TOL["bf16"], "Yg")
+    for name in ("U", "Bm", "Cm", "Delta", "Yg"):
+        assert_close(taps[name], im[name], TOL["bf16"], name)
     assert_close(out, ref, TOL["bf16"], "out")
+    return im
+
+
+@pytest.mark.parametrize("name", ["long_ctx", "zipf", "short_seqs"])
+def test_layer_full_size(name):
+    """Benchmark sizes on the "unit" recipe without the D skip: the scan output is then the state-space term alone
+    (share 1.0 of Y; on the N(0, 0.02^2) recipe it is ~1e-5 of Y and the D*u skip hides the recurrence, x Proj and
+    dt Proj from any relative tolerance), so S5, S6 and S7 are checked at full size, in the launch shapes bench.py
+    times (long_ctx: the chunked two-launch scan)."""
+    s = synth.CONFIGS[name]
+    _layer_full_size(s, synth.make_inputs(s, recipe="unit", with_D=False))
+
+
+def test_layer_full_size_benchmark_inputs():
+    """The very inputs bench.py times (N(0, 0.02^2) weights, D = 1): covers routing, in_proj, conv, gate, out_proj and the
+    skip term on those bits; the recurrence itself is invisible here and is covered by test_layer_full_size."""
+    s = synth.CONFIGS["long_ctx"]
+    _layer_full_size(s, synth.make_inputs(s))
+
+
+@pytest.mark.parametrize("B,L,De,disc_mode,use_ws", [
+    (1, 16384, 4096, 0, True),       # the launch bench.py --stage scan times: 10 chunks, two launches + state chain
+    (1, 16384, 4096, 1, True),
+    (64, 1024, 3072, 0, False),      # short_seqs shape: one pass, 8 states per thread
+])
+def test_scan_full_size(B, L, De, disc_mode, use_ws):
+    """rom_scan alone at benchmark sizes on O(1) inputs with an initial state, against the sequential fp64 recurrence:
+    y (gated, with skip) within 2e-2 and the final state within 2e-3."""
+    q = synth.make_scan_inputs(B, L, De, 16, "bf16", 9700 + L, with_z=True, with_h0=True)
+    cfg = rb.make_config(B, L, 64, De, 16, 4, 16, 1, 1, "bf16", 0, disc_mode)
+    d = {k: (None if v is None else v.cuda()) for k, v in q.items()}
+    y = torch.empty_like(d["u"])
+    h_last = torch.empty((B, De, 16), dtype=torch.float32, device="cuda")
+    ws = torch.empty(rb.scan_workspace_size(cfg), dtype=torch.uint8, device="cuda") if use_ws else None
+    rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], d["h0"], y, h_last, ws)
+    torch.cuda.synchronize()
+    got_y, got_h = np64(y), np64(h_last)
+    del d, y, h_last, ws
+    torch.cuda.empty_cache()
+    Y, hl = O.selective_scan(np64(q["u"]), np64(q["delta"]), np64(q["A"]), np64(q["Bm"]), np64(q["Cm"]), np64(q["D"]),
+                             np64(q["h0"]), disc_mode)
+    Y = O.gated(Y, np64(q["z"]))
+    assert_close(got_y, Y, TOL["bf16"], "scan y")
+    assert_close(got_h, hl, 2e-3, "scan h_last")
 
 
 def test_ffn_moe_full_size_sampled_tokens():
@@ -81,15 +130,7 @@ def test_layer_step_full_size():
 def test_layer_full_size_per_expert_small_projections():
     """The per-expert x Proj / dt Proj mode (`bench.py --small-proj routed`) at the benchmark workload."""
     s = synth.CONFIGS["long_ctx"]
-    p = synth.make_inputs(s, routed_small=True)
-    g = GpuLayer(s, p)
-    out = np64(g.forward())
-    idx = g.idx.cpu().numpy()
-    del g
-    torch.cuda.empty_cache()
-    ref, im = oracle_layer(s, p)
-    np.testing.assert_array_equal(idx, im["idx"])
-    assert_close(out, ref, TOL["bf16"], "out")
+    _layer_full_size(s, synth.make_inputs(s, recipe="unit", with_D=False, routed_small=True))
 
 
 @pytest.mark.parametrize("name", ["long_ctx", "zipf"])

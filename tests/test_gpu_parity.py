@@ -97,7 +97,7 @@ def run_scan(B, L, De, dtype, disc_mode, with_z, with_h0, with_D, seed, use_ws=F
     d = {k: (None if v is None else v.cuda()) for k, v in q.items()}
     y = torch.empty_like(d["u"])
     h_last = torch.empty((B, De, 16), dtype=torch.float32, device="cuda")
-    ws = rb.alloc_workspace(cfg) if use_ws else None      # with a workspace long sequences run as parallel chunks
+    ws = torch.empty(max(rb.scan_workspace_size(cfg), 16), dtype=torch.uint8, device="cuda") if use_ws else None      # with a workspace long sequences run as parallel chunks
     rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], d["h0"], y, h_last, ws)
     torch.cuda.synchronize()
     Y, hl = O.selective_scan(np64(q["u"]), np64(q["delta"]), np64(q["A"]), np64(q["Bm"]), np64(q["Cm"]), np64(q["D"]),
