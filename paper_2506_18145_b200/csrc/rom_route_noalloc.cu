@@ -77,14 +77,9 @@ extern "C" int rom_route_noalloc(const rom_config* cfg, const void* x, const voi
                                  int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
                                  int32_t* perm, int32_t* inv_perm, void* stream) {
   if (!cfg || !x || !W_r) return ROM_ERR_INVALID_ARG;
+  const int cfg_rc = check_config(cfg, 1);      // the same argument rules as rom_route
+  if (cfg_rc != ROM_OK) return cfg_rc;
   const rom_config& c = *cfg;
-  if (c.dtype != ROM_F32 && c.dtype != ROM_BF16) return ROM_ERR_INVALID_ARG;
-  if (c.B < 1 || c.L < 1 || c.E < 1 || c.K < 1 || c.K > c.E) return ROM_ERR_INVALID_ARG;
-  if (c.gate_mode != 0 && c.gate_mode != 1) return ROM_ERR_INVALID_ARG;
-  if (c.d_model < 64 || c.d_model % 64 != 0) return ROM_ERR_INVALID_ARG;
-  if ((c.flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
-  if (c.small_proj_experts != 0 && c.small_proj_experts != 1 && c.small_proj_experts != c.E) return ROM_ERR_INVALID_ARG;
-  if (c.E > kMaxE || c.K > kMaxK) return ROM_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(x) & 15u) || (reinterpret_cast<uintptr_t>(W_r) & 15u)) return ROM_ERR_INVALID_ARG;
   // the built-in scratch has a fixed size: larger problems must use rom_route with a caller workspace
   if ((int64_t)c.B * c.L > kNoAllocMaxTokens || (int64_t)c.B * c.L * c.K > kNoAllocMaxAssign) return ROM_ERR_STATIC_SCRATCH;

@@ -551,6 +551,21 @@ def test_load_balance_loss_uniform_router_value():
     assert abs(val0 - 1e-3 * E) < 1e-15   # collapse onto one expert is N times worse
 
 
+def test_load_balance_loss_top2_counts_every_dispatch():
+    """Top-2 with a uniform router: every token is dispatched to two experts, so F_i (tokens dispatched to i over all
+    tokens, Appendix A.3) is K/N, the F_i sum to K, and the value is alpha * N * sum_i (K/N)(1/N) = alpha * K.
+    Dividing by assignments instead of tokens would give alpha."""
+    T, E, K = 64, 8, 2
+    P = np.full((T, E), 1.0 / E)
+    idx = np.stack([np.arange(T) % E, (np.arange(T) + 3) % E], axis=1)
+    val, Fr = O.load_balance_loss(P, idx, alpha=1e-3)
+    np.testing.assert_allclose(Fr, K / E)
+    assert abs(Fr.sum() - K) < 1e-15 and abs(val - 1e-3 * K) < 1e-15
+    # a skewed softmax mean with the same dispatch: alpha * N * sum_i (K/N) Pbar_i = alpha * K again (Pbar sums to 1)
+    Ps = np.tile(np.linspace(1.0, 2.0, E) / np.linspace(1.0, 2.0, E).sum(), (T, 1))
+    assert abs(O.load_balance_loss(Ps, idx, alpha=1e-3)[0] - 1e-3 * K) < 1e-15
+
+
 # ---------------------------------------------------------------------------------------------- planted mistakes
 def test_pins_catch_planted_mistakes(monkeypatch):
     """Each planted bug (on the CPU, in the oracle) must break the dense-Mamba reduction."""
