@@ -6,7 +6,9 @@
  *
  * General rules
  *   - Every pointer is a DEVICE pointer unless marked "host".  The caller owns every buffer; the
- *     library allocates no device memory and keeps no state on the device between calls.
+ *     library allocates no device memory and keeps no state on the device between calls.  The one
+ *     exception is rom_route_noalloc: its scratch is an array resident in the library's device image, so
+ *     overlapping calls of it on one GPU must be serialised by the caller (see its own comment).
  *   - All tensors are dense, row-major, channels-last; device pointers must be 16-byte aligned.
  *   - "dtype" tensors are stored as ROM_F32 (float) or ROM_BF16 (bfloat16) as rom_config.dtype says.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream);
@@ -43,7 +45,9 @@ typedef enum {
   ROM_ERR_CUDA = -4,           /* a CUDA runtime/driver call failed (launch, tensor-map encode)   */
   ROM_ERR_ARCH = -5,           /* the current device is not sm_100                                */
   ROM_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait expired (reported by rom_get_status) */
-  ROM_ERR_STATIC_SCRATCH = -7  /* the problem does not fit the built-in scratch of rom_route_noalloc */
+  ROM_ERR_STATIC_SCRATCH = -7, /* the problem does not fit the built-in scratch of rom_route_noalloc */
+  ROM_ERR_DEBUG_CHECK = -8     /* ROM_FLAG_DEBUG_CHECKS: a routing-table index out of range or a workspace canary
+                                  overwritten (reported by rom_get_status)                          */
 } rom_status;
 
 typedef struct {
@@ -65,6 +69,18 @@ typedef struct {
 
 #define ROM_FLAG_SIMT_GEMM 1  /* run every projection on the plain fp32-FMA kernels (bisecting aid;
                                  always the case for ROM_F32) instead of the tcgen05 tensor path   */
+#define ROM_FLAG_DEBUG_CHECKS 2 /* rom_layer_forward / rom_layer_step only.  Every gather and scatter of the layer takes
+                                 its row index from the routing tables: they are validated on the device before any
+                                 kernel uses them (ranges, the two row <-> assignment maps agree, tile -> expert,
+                                 padded offsets), and 256-byte canaries between the workspace sub-buffers are written
+                                 before the first kernel and compared after the last.  A violation is latched as
+                                 ROM_ERR_DEBUG_CHECK.  The workspace is larger with this flag (rom_workspace_size and
+                                 rom_workspace_find take it into account); two more small launches per call.      */
+#define ROM_FLAG_TEST_STALL 4 /* fault injection for tests of the device-side timeout path (tensor path only): the
+                                 first grouped projection withholds the copies of one operand stage per CTA and
+                                 every device wait gives up after 2^14 polls instead of 2^22, so the call returns
+                                 normally, produces no valid output, and rom_get_status reports
+                                 ROM_ERR_DEVICE_TIMEOUT.  The workspace stays usable for the next call.          */
 
 typedef struct {                /* all read-only device pointers                                   */
   const void  *W_r;             /* [E, d_model]              dtype  router, W_r of Section 4.2 transposed */
@@ -157,6 +173,24 @@ ROM_API int rom_scan(const rom_config *cfg, const void *u, const float *delta, c
              const float *Bm, const float *Cm, const float *D, const void *z, const float *h0,
              void *y, float *h_last, void *ws, size_t ws_bytes, void *stream);
 
+/* Backward of rom_scan (Section 5.1 trains the layer end to end; the recurrence differentiated is that of Section
+ * 3.1): given dy = dLoss/d(output of rom_scan), the gradients of every input of the same call.
+ *   forward   h_t = a_t h_{t-1} + b_t u_t,  y_t = C_t h_t + D u_t,  out_t = y_t SiLU(z_t)  (a = exp(Delta A), b per disc_mode)
+ *   reverse   g = dLoss/dh_t:  g += C_t e_t (e = dy SiLU(z));  dC_t = sum_c e_t h_t;  da = g h_{t-1};  db = g u_t;  g <- a_t g
+ *   dy, u, z : [B, L, d_inner] dtype (z NULL = no gate);  delta : [B, L, d_inner] fp32;  A, Bm, Cm, D, h0 as in rom_scan;
+ *   dh_last  : [B, d_inner, d_state] fp32 or NULL: gradient arriving at the final state.
+ * Outputs: du, dz [B, L, d_inner] dtype (dz NULL exactly when z is);  ddelta [B, L, d_inner] fp32;  dA [d_inner, d_state],
+ *   dBm, dCm [B, L, d_state], dD [d_inner] (NULL exactly when D is) fp32, each the sum over everything that shares the
+ *   parameter (dA and dD over sequences and steps; dBm, dCm over channels) -- accumulated with floating-point atomics,
+ *   so their last bits vary from run to run;  dh0 [B, d_inner, d_state] fp32 or NULL.
+ * ws: rom_scan_backward_workspace_size(cfg) bytes (the state at the start of every 32 steps).  All arithmetic fp32.
+ * Uses cfg->B, L, d_inner, d_state, dtype, disc_mode.                                                              */
+ROM_API int rom_scan_backward_workspace_size(const rom_config *cfg, size_t *bytes);
+ROM_API int rom_scan_backward(const rom_config *cfg, const void *dy, const void *u, const float *delta, const float *A,
+                      const float *Bm, const float *Cm, const float *D, const void *z, const float *h0,
+                      const float *dh_last, void *du, float *ddelta, float *dA, float *dBm, float *dCm, float *dD,
+                      void *dz, float *dh0, void *ws, size_t ws_bytes, void *stream);
+
 /* Forward pass of one RoM layer (Section 4.2 equations for G, H_t, O_t, E_i with the shared
  * Conv1D / x Proj / dt Proj / A / D of Section 4.3):
  *   route -> gather tokens by expert -> per-expert [Conv Proj | Gate Proj] -> un-permute, sum over
@@ -233,9 +267,16 @@ ROM_API const char *rom_stage_name(int i);
  * Returns ROM_ERR_INVALID_ARG for an unknown name.                                                */
 ROM_API int rom_workspace_find(const rom_config *cfg, const char *name, size_t *offset, size_t *bytes);
 
+/* Re-run the checks of ROM_FLAG_DEBUG_CHECKS on a workspace that the last rom_layer_forward / rom_layer_step call
+ * with that flag (same cfg) has filled: routing tables and canaries (a debugging aid; the paper has no counterpart).
+ * Asynchronous on `stream`; the verdict is read with rom_get_status.  cfg->flags must carry the flag.  */
+ROM_API int rom_debug_check(const rom_config *cfg, void *ws, size_t ws_bytes, void *stream);
+
 /* Read and clear the device status word of a workspace.  `host_code` (host out) receives ROM_OK or the
  * rom_status a kernel latched: ROM_ERR_DEVICE_TIMEOUT (a bounded wait expired) or ROM_ERR_INVALID_ARG
- * (rom_ffn_moe_forward met an expert index out of range).  This call synchronises `stream`.       */
+ * (rom_ffn_moe_forward met an expert index out of range) or ROM_ERR_DEBUG_CHECK (ROM_FLAG_DEBUG_CHECKS; the second
+ * and third int32 of the workspace then hold which check failed -- 10..15 a routing table, 20 a canary -- and the
+ * offending index, until this call clears them).  This call synchronises `stream`.                  */
 ROM_API int rom_get_status(void *ws, void *stream, int32_t *host_code);
 
 /* Static string for a rom_status value.                                                           */

@@ -17,13 +17,15 @@ LIB_PATH = os.path.join(_PKG, "librom_b200.so")
 
 ROM_F32, ROM_BF16 = 0, 1
 ROM_FLAG_SIMT_GEMM = 1
+ROM_FLAG_DEBUG_CHECKS = 2
+ROM_FLAG_TEST_STALL = 4
 ROM_OK = 0
 
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
            "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance",
            "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step", "rom_layer_forward_host",
-           "rom_scan_workspace_size")
+           "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward")
 
 
 class RomConfig(ctypes.Structure):
@@ -58,6 +60,9 @@ def lib() -> ctypes.CDLL:
         cfgp = ctypes.POINTER(RomConfig)
         L.rom_workspace_size.argtypes = [cfgp, szp]
         L.rom_scan_workspace_size.argtypes = [cfgp, szp]
+        L.rom_debug_check.argtypes = [cfgp, vp, ctypes.c_size_t, vp]
+        L.rom_scan_backward_workspace_size.argtypes = [cfgp, szp]
+        L.rom_scan_backward.argtypes = [cfgp] + [vp] * 19 + [ctypes.c_size_t, vp]
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
         L.rom_route_noalloc.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
         L.rom_route_balance.argtypes = [cfgp, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp, ctypes.c_size_t, vp]
@@ -126,7 +131,7 @@ def scan_workspace_size(cfg: RomConfig) -> int:
     n = ctypes.c_size_t(0)
     rc = lib().rom_scan_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
     if rc != ROM_OK:
-        raise RomError(rc, "rom_scan_workspace_size")
+        raise RomError(rc, "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward")
     return int(n.value)
 
 
@@ -176,6 +181,24 @@ def rom_scan(cfg, u, delta, A, Bm, Cm, D, z, h0, y, h_last, ws=None, stream=None
     return rc
 
 
+def scan_backward_workspace_size(cfg: RomConfig) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().rom_scan_backward_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_scan_backward_workspace_size")
+    return int(n.value)
+
+
+def rom_scan_backward(cfg, dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0, ws,
+                      stream=None, check=True) -> int:
+    rc = lib().rom_scan_backward(ctypes.byref(cfg), _ptr(dy), _ptr(u), _ptr(delta), _ptr(A), _ptr(Bm), _ptr(Cm), _ptr(D), _ptr(z),
+                                 _ptr(h0), _ptr(dh_last), _ptr(du), _ptr(ddelta), _ptr(dA), _ptr(dBm), _ptr(dCm), _ptr(dD),
+                                 _ptr(dz), _ptr(dh0), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_scan_backward")
+    return rc
+
+
 def make_weights(w: Dict[str, Optional[torch.Tensor]]) -> RomWeights:
     return RomWeights(*[_ptr(w.get(n)) for n, _ in RomWeights._fields_])
 
@@ -218,6 +241,13 @@ def rom_layer_step(cfg, weights: RomWeights, x, conv_state, ssm_state, out, topk
                               _ptr(topk_idx_out), _ptr(gates_out), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_layer_step")
+    return rc
+
+
+def rom_debug_check(cfg, ws, stream=None, check=True) -> int:
+    rc = lib().rom_debug_check(ctypes.byref(cfg), _ptr(ws), ws.numel(), _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_debug_check")
     return rc
 
 

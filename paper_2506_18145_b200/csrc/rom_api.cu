@@ -18,7 +18,13 @@ WsLayout make_layout(const rom_config& c) {
   l.n_chunks = (l.T + kChunkTokens - 1) / kChunkTokens;
   const int R = c.dt_rank, N = c.d_state;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  const bool canaries = (c.flags & ROM_FLAG_DEBUG_CHECKS) != 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o = align_up(o + bytes, 256);
+    if (canaries && l.n_canary < kMaxCanaries) { l.canary[l.n_canary++] = o; o += kCanaryBytes; }
+    return at;
+  };
   l.status = take(sizeof(int32_t) * kStatusInts);
   l.counts = take(sizeof(int32_t) * c.E);
   l.offsets = take(sizeof(int32_t) * (c.E + 1));
@@ -55,16 +61,27 @@ WsLayout make_layout(const rom_config& c) {
   return l;
 }
 
-namespace {
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+cudaError_t current_device_sm_count(int* n) {
+  constexpr int kMaxDev = 64;
+  static int cache[kMaxDev] = {};      // 0 = not looked up yet; every writer stores the same value for a device
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < kMaxDev && cache[dev] > 0) { *n = cache[dev]; return cudaSuccess; }
+  int v = 0;
+  e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  if (dev >= 0 && dev < kMaxDev) cache[dev] = v;
+  *n = v;
+  return cudaSuccess;
+}
 
 // which == 0: full layer; 1: route only; 2: scan only
 int check_config(const rom_config* c, int which) {
   if (!c) return ROM_ERR_INVALID_ARG;
   if (c->dtype != ROM_F32 && c->dtype != ROM_BF16) return ROM_ERR_INVALID_ARG;
   if (c->B < 1 || c->L < 1) return ROM_ERR_INVALID_ARG;
-  if ((c->flags & ~ROM_FLAG_SIMT_GEMM) != 0) return ROM_ERR_INVALID_ARG;
+  if ((c->flags & ~(ROM_FLAG_SIMT_GEMM | ROM_FLAG_DEBUG_CHECKS | ROM_FLAG_TEST_STALL)) != 0) return ROM_ERR_INVALID_ARG;
   if (which != 2) {
     if (c->E < 1 || c->K < 1 || c->K > c->E) return ROM_ERR_INVALID_ARG;
     if (c->E > kMaxE || c->K > kMaxK) return ROM_ERR_UNSUPPORTED;
@@ -91,6 +108,10 @@ int check_config(const rom_config* c, int which) {
   }
   return ROM_OK;
 }
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_device() {
   int dev = 0;
@@ -202,6 +223,33 @@ int rom_scan(const rom_config* cfg, const void* u, const float* delta, const flo
   return ROM_OK;
 }
 
+int rom_scan_backward_workspace_size(const rom_config* cfg, size_t* bytes) {
+  if (!bytes) return ROM_ERR_INVALID_ARG;
+  const int rc = check_config(cfg, 2);
+  if (rc != ROM_OK) return rc;
+  *bytes = scan_bwd_ws_bytes(cfg->B, cfg->d_inner, cfg->L);
+  return ROM_OK;
+}
+
+int rom_scan_backward(const rom_config* cfg, const void* dy, const void* u, const float* delta, const float* A, const float* Bm,
+                      const float* Cm, const float* D, const void* z, const float* h0, const float* dh_last, void* du,
+                      float* ddelta, float* dA, float* dBm, float* dCm, float* dD, void* dz, float* dh0, void* ws, size_t ws_bytes,
+                      void* stream) {
+  int rc = check_config(cfg, 2);
+  if (rc != ROM_OK) return rc;
+  if (!dy || !u || !delta || !A || !Bm || !Cm || !du || !ddelta || !dA || !dBm || !dCm || !ws) return ROM_ERR_INVALID_ARG;
+  if ((D == nullptr) != (dD == nullptr) || (z == nullptr) != (dz == nullptr)) return ROM_ERR_INVALID_ARG;
+  const void* ptrs[] = {dy, u, delta, A, Bm, Cm, du, ddelta, dA, dBm, dCm, ws, z, dz, h0, dh_last, dh0};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return ROM_ERR_INVALID_ARG;
+  if (ws_bytes < scan_bwd_ws_bytes(cfg->B, cfg->d_inner, cfg->L)) return ROM_ERR_WORKSPACE;
+  if ((rc = check_device()) != ROM_OK) return rc;
+  LaunchCounter::count = 0;
+  ROM_CUDA(launch_scan_backward(*cfg, dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0,
+                                static_cast<float*>(ws), static_cast<cudaStream_t>(stream)));
+  return ROM_OK;
+}
+
 }  // extern "C"
 
 namespace rom {
@@ -248,8 +296,11 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   } while (0)
   if (ev) ROM_CUDA(cudaEventRecord(ev[0], st));
   ROM_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t) * kStatusInts, st));
+  const bool debug_checks = (c.flags & ROM_FLAG_DEBUG_CHECKS) != 0;
+  if (debug_checks) ROM_CUDA(launch_canaries(W, lay, false, st));
   // S1 + S2: router, top-K, permutation tables
   ROM_CUDA(launch_route(c, x, w->W_r, w->b_r, topk_idx_out, gates, counts_out, nullptr, nullptr, nullptr, W, lay, st));
+  if (debug_checks) ROM_CUDA(launch_check_tables(c, W, lay, st));
   ROM_STAGE_DONE();
   ROM_CUDA(launch_gather_rows(c, x, W, lay, st));
   ROM_STAGE_DONE();
@@ -260,7 +311,8 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
     // single CTA; the lane-split kernel spreads it over the GPU
     if (!te && M_max <= 128 && Kd >= 1024 && Kd % 2048 == 0 && ep.mode == EPI_XPROJ)
       return launch_gemm_skinny(c.dtype, A_, lda, B_, ldb, M_max, Nn, Kd, ep, st);
-    if (tc) return launch_gemm_tc(A_, lda, B_, ldb, n_experts, M_max, Nn, Kd, te, nmt, ep, status, st);
+    if (tc) return launch_gemm_tc(A_, lda, B_, ldb, n_experts, M_max, Nn, Kd, te, nmt, ep, status, st,
+                                  (c.flags & ROM_FLAG_TEST_STALL) != 0 && (ep.mode == EPI_INPROJ || (ep.mode == EPI_STORE && Nn == 2 * De)));
     return launch_gemm_simt(c.dtype, A_, lda, B_, ldb, bstride, M_max, Nn, Kd, te, nmt, ep, st);
   };
 
@@ -339,6 +391,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
     ROM_STAGE_DONE();
   }
 #undef ROM_STAGE_DONE
+  if (debug_checks) ROM_CUDA(launch_canaries(W, lay, true, st));
   return ROM_OK;
 }
 
@@ -390,6 +443,19 @@ int rom_layer_forward_profile(const rom_config* cfg, const rom_weights* w, const
   return rc;
 }
 
+int rom_debug_check(const rom_config* cfg, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg, 0);
+  if (rc != ROM_OK) return rc;
+  if (!(cfg->flags & ROM_FLAG_DEBUG_CHECKS)) return ROM_ERR_INVALID_ARG;
+  if (!ws || !aligned16(ws)) return ROM_ERR_INVALID_ARG;
+  const WsLayout lay = make_layout(*cfg);
+  if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ROM_CUDA(launch_check_tables(*cfg, static_cast<char*>(ws), lay, st));
+  ROM_CUDA(launch_canaries(static_cast<char*>(ws), lay, true, st));
+  return ROM_OK;
+}
+
 int rom_num_stages(void) { return kNumStages; }
 
 const char* rom_stage_name(int i) { return (i >= 0 && i < kNumStages) ? kStageNames[i] : ""; }
@@ -415,6 +481,7 @@ const char* rom_status_string(int code) {
     case ROM_ERR_ARCH: return "device is not sm_100";
     case ROM_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
     case ROM_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch of rom_route_noalloc";
+    case ROM_ERR_DEBUG_CHECK: return "a debug check failed (routing-table index out of range or workspace canary overwritten)";
     default: return "unknown status";
   }
 }

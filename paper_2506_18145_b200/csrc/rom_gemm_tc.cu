@@ -16,7 +16,8 @@
 //               chunks, and the load of the next chunk is in flight while one chunk is processed
 // The accumulator is double-buffered in TMEM (2 x 256 columns) so the epilogue of tile i overlaps
 // the MMAs of tile i+1.  Every mbarrier wait is bounded; on expiry the CTA latches an error code in
-// the status word, drains its own copies with a bounded wait, frees its TMEM and returns.
+// the status word, waits (bounded) for its own copies and for the MMAs it already issued, frees its
+// TMEM and returns.
 //
 // Every TMA load here is a plain single-CTA load (no thread-block clusters).
 #include <cuda.h>
@@ -58,7 +59,8 @@ __host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(
 __host__ __device__ constexpr int smem_bytes_of(int mode) {
   return stages_of(mode) * stage_bytes_of(mode) + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
 }
-constexpr uint32_t WAIT_LIMIT = 1u << 22;   // try_wait polls before a wait gives up (a few seconds)
+constexpr uint32_t WAIT_LIMIT = 1u << 22;        // try_wait polls before a wait gives up (a few seconds)
+constexpr uint32_t WAIT_LIMIT_TEST = 1u << 14;   // the same under the fault-injection flag (milliseconds)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -81,8 +83,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the limit is reached or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *abort_flag) return false;
   }
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M_max, int N, int Kd, int block_n, uint32_t idesc,
                const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ num_m_tiles_dev,
-               Epilogue ep, int32_t* __restrict__ status) {
+               Epilogue ep, int32_t* __restrict__ status, uint32_t wait_limit, int withhold_kb) {
   constexpr int STAGES = stages_of(MODE);
   constexpr int SB = stage_bytes_of(MODE);          // bytes per operand stage (multiple of 1024)
   extern __shared__ unsigned char smem_raw[];
@@ -295,7 +297,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + ACC_STAGES + a); };
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + STAGES * SB + 8 * (2 * STAGES + 2 * ACC_STAGES));
+  const uint32_t drain_bar = bars + 8u * (2 * STAGES + 2 * ACC_STAGES);      // abort path only: completion of the MMAs already issued
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + STAGES * SB + 8 * (2 * STAGES + 2 * ACC_STAGES + 1));
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   float* out_stage = reinterpret_cast<float*>(smem + STAGES * SB + 256);        // [8 warps][32][32] (softplus only)
 
@@ -313,6 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), epi_warps_of(MODE)); }
+    mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -337,13 +341,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int e = tile_expert ? tile_expert[m_tile] : 0;
         const int b_row = MODE == EPI_SWIGLU ? e * 2 * N + n_tile * 128 : e * N + n_tile * block_n;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), stage_tx);
           const uint32_t sa = base + stage * SB;
-          tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BLOCK_K, m_tile * BLOCK_M);
-          tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row);
-          if (MODE == EPI_SWIGLU)     // second half of the B tile: the up rows of the same 128 hidden units (box = 128 rows)
-            tma_load_2d(sa + A_STAGE_BYTES + 128 * BLOCK_K * 2, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row + N);
+          // fault injection (tests only): the copies of K block `withhold_kb` of this CTA's first tile are never issued,
+          // so the stage never fills and the waits downstream run out
+          if (!(withhold_kb >= 0 && tile == (int)blockIdx.x && kb == withhold_kb)) {
+            tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BLOCK_K, m_tile * BLOCK_M);
+            tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row);
+            if (MODE == EPI_SWIGLU)     // second half of the B tile: the up rows of the same 128 hidden units (box = 128 rows)
+              tma_load_2d(sa + A_STAGE_BYTES + 128 * BLOCK_K * 2, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row + N);
+          }
           ++issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -357,7 +365,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         int s = stage; uint32_t ph = phase;
         for (int i = 0; i < min(issued, STAGES); ++i) {
           if (--s < 0) { s = STAGES - 1; ph ^= 1u; }
-          for (uint32_t it = 0; it < (1u << 20); ++it)
+          for (uint32_t it = 0; it < (wait_limit >> 2); ++it)
             if (mbar_try_wait(full_bar(s), ph)) break;
         }
       }
@@ -367,13 +375,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      bool ok = true;
+      bool ok = true, issued_any = false;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)acc * MAX_BLOCK_N;
         for (int kb = 0; kb < num_kb; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, wait_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * SB;
           const uint64_t adesc = make_smem_desc(sa);
@@ -384,6 +392,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             umma_bf16(tmem_d, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0 ? 1u : 0u);
           }
           umma_commit(empty_bar(stage));
+          issued_any = true;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
@@ -393,6 +402,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!ok) {
         if (!*abort_flag) { atomicExch(status + kStatCode, ROM_ERR_DEVICE_TIMEOUT); atomicExch(status + kStatWhere, 2); }
         *abort_flag = 1;
+      }
+      if (*abort_flag && issued_any) {
+        // the MMAs already issued may still read shared memory and write tensor memory: one more commit tracks them
+        // all; wait for it (bounded) before the CTA frees its tensor memory
+        umma_commit(drain_bar);
+        for (uint32_t it = 0; it < (wait_limit >> 2); ++it)
+          if (mbar_try_wait(drain_bar, 0)) break;
       }
     }
   } else {
@@ -405,7 +421,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const int m_tile = tile / n_tiles, n_tile = tile % n_tiles;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      // warp-uniform outcome: the tensor-memory loads below need the whole warp
+      if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, wait_limit))) { ok = false; break; }
       tc_fence_after();
       const int row = m_tile * BLOCK_M + quarter * 32 + lane;
       bool row_ok = row < M_valid;
@@ -543,7 +560,7 @@ bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
 
 cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int n_experts, int M_max, int N, int Kd,
                            const int32_t* tile_expert, const int32_t* num_m_tiles_dev, const Epilogue& epi,
-                           int32_t* status, cudaStream_t st) {
+                           int32_t* status, cudaStream_t st, bool test_stall) {
   // N tile: a multiple of 32 (epilogue column groups) and of 16 (UMMA N for M = 128), at most 256
   const bool swiglu = epi.mode == EPI_SWIGLU;      // N output columns from 2N rows of B per expert, loaded as two boxes of 128 rows
   if (swiglu && (N % 128 != 0 || MAX_BLOCK_N != 256)) return cudaErrorInvalidValue;
@@ -555,26 +572,22 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
     return cudaErrorInvalidValue;
   // instruction descriptor: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
   const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-  }
+  int num_sms = 0;
+  cudaError_t e = current_device_sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
   auto kern = epi.mode == EPI_STORE ? gemm_tc_kernel<EPI_STORE> : epi.mode == EPI_XPROJ ? gemm_tc_kernel<EPI_XPROJ>
               : epi.mode == EPI_INPROJ ? gemm_tc_kernel<EPI_INPROJ> : epi.mode == EPI_OUTPROJ ? gemm_tc_kernel<EPI_OUTPROJ>
               : epi.mode == EPI_F32 ? gemm_tc_kernel<EPI_F32> : epi.mode == EPI_SWIGLU ? gemm_tc_kernel<EPI_SWIGLU>
               : epi.mode == EPI_SOFTPLUS_ROWS ? gemm_tc_kernel<EPI_SOFTPLUS_ROWS>
               : gemm_tc_kernel<EPI_SOFTPLUS>;
   const int smem_bytes = smem_bytes_of(epi.mode);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
   if (e != cudaSuccess) return e;
   const int n_tiles = swiglu ? N / 128 : (N + block_n - 1) / block_n;
   const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
   const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
-  kern<<<grid, threads_of(epi.mode), smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status);
+  kern<<<grid, threads_of(epi.mode), smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status,
+                                                            test_stall ? WAIT_LIMIT_TEST : WAIT_LIMIT, test_stall ? 1 : -1);
   count_launch();
   return cudaGetLastError();
 }

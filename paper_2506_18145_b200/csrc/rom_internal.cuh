@@ -17,7 +17,10 @@ constexpr int kStatusInts = 64;    // status block at the head of the workspace
 
 // status word slots
 constexpr int kStatCode = 0;       // 0 or the rom_status a kernel latched (a wait that expired, an index out of range)
-constexpr int kStatWhere = 1;      // which wait gave up (debug aid)
+constexpr int kStatWhere = 1;      // which wait gave up / which debug check failed (debug aid)
+constexpr int kStatIndex = 2;      // debug checks: the offending index
+constexpr int kMaxCanaries = 40;   // sub-buffers of the workspace (debug checks put a canary after each)
+constexpr int kCanaryBytes = 256;
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -53,8 +56,21 @@ struct WsLayout {
   size_t total;
   int64_t T, A, rows_max, max_m_tiles, n_chunks;
   size_t esz;
+  size_t canary[kMaxCanaries];        // ROM_FLAG_DEBUG_CHECKS: offset of the canary after each sub-buffer
+  int n_canary;
 };
 WsLayout make_layout(const rom_config& c);
+
+// Host-side checks of a rom_config shared by every entry point.  which == 0: full layer; 1: route only; 2: scan only.
+int check_config(const rom_config* c, int which);
+
+// Number of SMs of the current device (looked up per device ordinal; nothing is assumed about other devices).
+cudaError_t current_device_sm_count(int* n);
+
+// ROM_FLAG_DEBUG_CHECKS: validate the routing tables in the workspace (latches ROM_ERR_DEBUG_CHECK in the status word);
+// write (check == false) or compare (check == true) the canary words between the workspace sub-buffers.
+cudaError_t launch_check_tables(const rom_config& c, char* ws, const WsLayout& lay, cudaStream_t st);
+cudaError_t launch_canaries(char* ws, const WsLayout& lay, bool check, cudaStream_t st);
 
 struct LaunchCounter { static thread_local int count; };
 inline void count_launch() { LaunchCounter::count++; }
@@ -126,7 +142,7 @@ cudaError_t launch_gemm_skinny(int dtype, const void* A, int lda, const void* Bw
 
 cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int n_experts,
                            int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
-                           const Epilogue& epi, int32_t* status, cudaStream_t st);
+                           const Epilogue& epi, int32_t* status, cudaStream_t st, bool test_stall = false);
 
 // row_of_assign == nullptr (top-1, rows already in token order): row t of XZp belongs to token t.
 // Zs (K > 1 only): [T, d_inner], SiLU of the Gate Proj rows summed over the K slots.
@@ -147,6 +163,14 @@ cudaError_t launch_conv_step(const rom_config& c, const void* XZp, const int32_t
 cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
                         void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st);
+
+// Backward of the scan (gradients of every input); ckpt: scan_bwd_ws_bytes() bytes of scratch.  dA, dBm, dCm, dD are
+// zeroed here and accumulated with atomics.  z / dz, h0, dh_last, dD, dh0 may be null.
+size_t scan_bwd_ws_bytes(int B, int De, int L);
+cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void* u, const float* delta, const float* A,
+                                 const float* Bm, const float* Cm, const float* D, const void* z, const float* h0,
+                                 const float* dh_last, void* du, float* ddelta, float* dA, float* dBm, float* dCm, float* dD,
+                                 void* dz, float* dh0, float* ckpt, cudaStream_t st);
 
 cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,
                            void* out, cudaStream_t st);

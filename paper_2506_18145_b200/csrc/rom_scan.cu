@@ -563,14 +563,9 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
 cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
                         void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st) {
-  static int num_sms = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return e;
-  }
+  int num_sms = 0;
+  const cudaError_t e = current_device_sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
   const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0};
   if (c.dtype != ROM_BF16) return launch_scan_t<float, float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
   return delta_fp32 ? launch_scan_t<__nv_bfloat16, float, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)

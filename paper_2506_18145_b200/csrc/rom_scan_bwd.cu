@@ -1,0 +1,276 @@
+// Backward of the selective scan (Section 3.1 recurrence; Section 5.1 trains the layer end to end).
+//
+// Forward:  h_t = a_t h_{t-1} + b_t u_t,  y_t = sum_n C_t,n h_t,n + D u_t,  out_t = y_t * SiLU(z_t)   (gate optional)
+//           a = exp(Delta A);  b = expm1(Delta A)/A * B (zero-order hold)  or  Delta B.
+// Reverse, with g = dLoss/dh_t carried from later steps and e_t = dout_t * SiLU(z_t):
+//           g += C_t e_t;  dC_t = sum_c e_t h_t;  dA-bar = g h_{t-1};  db = g u_t;  du_t = sum_n g b + D e_t;  g <- a_t g.
+//
+// The reverse sweep needs h_{t-1} and h_t at every step.  A first kernel runs the recurrence forward and keeps the
+// state at the start of every chunk of 32 steps (checkpoints in the workspace).  The second kernel walks the chunks
+// backwards: it recomputes the chunk's states from its checkpoint into shared memory, then sweeps the chunk in
+// reverse.  A thread owns 4 of the 16 states of one channel of one sequence (4 adjacent lanes per channel): sums over
+// the states (dDelta, du, the forward y for the gate's derivative) are shuffles over those lanes; sums over channels
+// (dB, dC) are shuffles over the 8 channels of a warp, shared-memory atomics over the block and one global atomic per
+// (step, state) and block; dA and dD accumulate in registers over the sequence and leave with one atomic per thread.
+// All arithmetic is fp32 with the accurate exp / expm1 (both storage types): this is the first, plain version of
+// the kernel; its time is not tuned.
+#include "rom_internal.cuh"
+
+namespace rom {
+namespace {
+
+constexpr int NST = 16;
+constexpr int CK = 32;            // steps per chunk
+constexpr int BCH = 32;           // channels per block
+constexpr int BT = BCH * 4;       // threads per block
+constexpr size_t BWD_SMEM = sizeof(float4) * CK * BT + sizeof(float) * CK * (8 * BCH + 4 * NST);
+
+struct BwdArgs {
+  const void* dy; const void* u; const float* delta; const float* A; const float* Bm; const float* Cm; const float* D;
+  const void* z; const float* h0; const float* dh_last;
+  void* du; float* ddelta; float* dA; float* dBm; float* dCm; float* dD; void* dz; float* dh0;
+  float* ckpt;        // [B, nck, De, 16]
+  int L, De, nck;
+};
+
+__device__ __forceinline__ float sigmoid_f(float v) { return 1.0f / (1.0f + expf(-v)); }
+
+// Forward pass that only records the state at the start of every chunk.
+template <typename T, bool ZOH>
+__global__ void __launch_bounds__(BT)
+scan_ckpt_kernel(const BwdArgs p) {
+  const int tid = threadIdx.x, cl = tid >> 2, q = tid & 3;
+  const int c = blockIdx.x * BCH + cl;
+  const size_t b = blockIdx.y;
+  if (c >= p.De) return;
+  const T* __restrict__ u = static_cast<const T*>(p.u);
+  float a[4], h[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a[i] = p.A[(size_t)c * NST + 4 * q + i];
+    h[i] = p.h0 ? p.h0[(b * p.De + c) * NST + 4 * q + i] : 0.0f;
+  }
+  for (int t = 0; t < p.L; ++t) {
+    if ((t % CK) == 0)
+      *reinterpret_cast<float4*>(p.ckpt + ((b * p.nck + t / CK) * p.De + c) * NST + 4 * q) = make_float4(h[0], h[1], h[2], h[3]);
+    const size_t e = (b * p.L + t) * p.De + c;
+    const float dl = p.delta[e], uu = to_f32(u[e]);
+    const float4 B4 = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
+    const float bv[4] = {B4.x, B4.y, B4.z, B4.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float x = dl * a[i];
+      const float bb = ZOH ? expm1f(x) / a[i] * bv[i] : dl * bv[i];
+      h[i] = fmaf(expf(x), h[i], bb * uu);
+    }
+  }
+}
+
+template <typename T, bool ZOH>
+__global__ void __launch_bounds__(BT)
+scan_bwd_kernel(const BwdArgs p) {
+  extern __shared__ __align__(16) unsigned char bwd_smem[];
+  float4 (*hbuf)[BT] = reinterpret_cast<float4 (*)[BT]>(bwd_smem);                    // states after each step of the chunk (this thread's 4)
+  float (*s_dl)[BCH] = reinterpret_cast<float (*)[BCH]>(bwd_smem + sizeof(float4) * CK * BT);
+  float (*s_u)[BCH] = s_dl + CK;
+  float (*s_e)[BCH] = s_u + CK;
+  float (*s_z)[BCH] = s_e + CK;
+  float (*s_dy)[BCH] = s_z + CK;
+  float (*s_dd)[BCH] = s_dy + CK;
+  float (*s_du)[BCH] = s_dd + CK;
+  float (*s_y)[BCH] = s_du + CK;
+  float (*s_B)[NST] = reinterpret_cast<float (*)[NST]>(s_y + CK);
+  float (*s_C)[NST] = s_B + CK;
+  float (*s_dB)[NST] = s_C + CK;
+  float (*s_dC)[NST] = s_dB + CK;
+
+  const int tid = threadIdx.x, cl = tid >> 2, q = tid & 3, lane = tid & 31;
+  const int c_base = blockIdx.x * BCH;
+  const int c = c_base + cl;
+  const bool c_ok = c < p.De;
+  const int cc = c_ok ? c : p.De - 1;
+  const size_t b = blockIdx.y;
+  const T* __restrict__ u = static_cast<const T*>(p.u);
+  const T* __restrict__ dy = static_cast<const T*>(p.dy);
+  const T* __restrict__ z = static_cast<const T*>(p.z);
+  T* __restrict__ du = static_cast<T*>(p.du);
+  T* __restrict__ dz = static_cast<T*>(p.dz);
+
+  float a[4], g[4], dAacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a[i] = p.A[(size_t)cc * NST + 4 * q + i];
+    g[i] = p.dh_last ? p.dh_last[(b * p.De + cc) * NST + 4 * q + i] : 0.0f;
+  }
+  const float Dc = p.D ? p.D[cc] : 0.0f;
+  float dDacc = 0.0f;
+
+  for (int k = p.nck - 1; k >= 0; --k) {
+    const int t0 = k * CK;
+    const int nt = min(CK, p.L - t0);
+    // ---- stage the chunk's inputs; e = dout * SiLU(z) is the gradient arriving at y
+    for (int i = tid; i < CK * BCH; i += BT) {
+      const int r = i / BCH, j = i % BCH;
+      float dl = 0.0f, uu = 0.0f, dyv = 0.0f, zz = 0.0f;
+      if (r < nt && c_base + j < p.De) {
+        const size_t e = (b * p.L + t0 + r) * p.De + c_base + j;
+        dl = p.delta[e]; uu = to_f32(u[e]); dyv = to_f32(dy[e]);
+        if (z) zz = to_f32(z[e]);
+      }
+      s_dl[r][j] = dl; s_u[r][j] = uu; s_dy[r][j] = dyv; s_z[r][j] = zz;
+      s_e[r][j] = z ? dyv * zz * sigmoid_f(zz) : dyv;
+    }
+    for (int i = tid; i < CK * NST; i += BT) {
+      const int r = i / NST, n = i % NST;
+      const bool in = r < nt;
+      s_B[r][n] = in ? p.Bm[(b * p.L + t0 + r) * NST + n] : 0.0f;
+      s_C[r][n] = in ? p.Cm[(b * p.L + t0 + r) * NST + n] : 0.0f;
+      s_dB[r][n] = 0.0f; s_dC[r][n] = 0.0f;
+    }
+    __syncthreads();
+
+    // ---- recompute the chunk's states from its checkpoint
+    const float4 h4 = *reinterpret_cast<const float4*>(p.ckpt + ((b * p.nck + k) * p.De + cc) * NST + 4 * q);
+    const float hstart[4] = {h4.x, h4.y, h4.z, h4.w};
+    float h[4] = {h4.x, h4.y, h4.z, h4.w};
+    for (int r = 0; r < nt; ++r) {
+      const float dl = s_dl[r][cl], uu = s_u[r][cl];
+      float ys = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float x = dl * a[i];
+        const float bb = ZOH ? expm1f(x) / a[i] * s_B[r][4 * q + i] : dl * s_B[r][4 * q + i];
+        h[i] = fmaf(expf(x), h[i], bb * uu);
+        ys = fmaf(s_C[r][4 * q + i], h[i], ys);
+      }
+      hbuf[r][tid] = make_float4(h[0], h[1], h[2], h[3]);
+      if (z) {                                     // forward y (before the gate) for the gate's derivative
+        ys += __shfl_xor_sync(0xffffffffu, ys, 1);
+        ys += __shfl_xor_sync(0xffffffffu, ys, 2);
+        if (q == 0) s_y[r][cl] = fmaf(Dc, uu, ys);
+      }
+    }
+
+    // ---- reverse sweep over the chunk
+    for (int r = nt - 1; r >= 0; --r) {
+      const float dl = s_dl[r][cl], uu = s_u[r][cl], ev = c_ok ? s_e[r][cl] : 0.0f;
+      const float4 hc4 = hbuf[r][tid];
+      const float hc[4] = {hc4.x, hc4.y, hc4.z, hc4.w};
+      float hp[4];
+      if (r > 0) { const float4 v = hbuf[r - 1][tid]; hp[0] = v.x; hp[1] = v.y; hp[2] = v.z; hp[3] = v.w; }
+      else { hp[0] = hstart[0]; hp[1] = hstart[1]; hp[2] = hstart[2]; hp[3] = hstart[3]; }
+      float dd = 0.0f, duv = 0.0f, dBp[4], dCp[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float Bv = s_B[r][4 * q + i], Cv = s_C[r][4 * q + i];
+        g[i] = fmaf(Cv, ev, g[i]);
+        dCp[i] = ev * hc[i];
+        const float x = dl * a[i], ex = expf(x);
+        float dx = g[i] * hp[i] * ex;              // through A-bar = exp(x)
+        if (ZOH) {
+          const float em1 = expm1f(x), ia = 1.0f / a[i];
+          dx = fmaf(g[i] * uu * Bv * ia, ex, dx);  // through expm1(x)
+          dAacc[i] = fmaf(g[i] * uu * Bv, -em1 * ia * ia, dAacc[i]);
+          dBp[i] = g[i] * uu * em1 * ia;
+          duv = fmaf(g[i] * em1 * ia, Bv, duv);
+          dd = fmaf(dx, a[i], dd);
+        } else {
+          dBp[i] = g[i] * uu * dl;
+          duv = fmaf(g[i] * dl, Bv, duv);
+          dd = fmaf(dx, a[i], dd);
+          dd = fmaf(g[i] * uu, Bv, dd);
+        }
+        dAacc[i] = fmaf(dx, dl, dAacc[i]);
+        g[i] *= ex;
+      }
+      // sums over the 16 states: the 4 lanes of the channel
+      dd += __shfl_xor_sync(0xffffffffu, dd, 1);  dd += __shfl_xor_sync(0xffffffffu, dd, 2);
+      duv += __shfl_xor_sync(0xffffffffu, duv, 1); duv += __shfl_xor_sync(0xffffffffu, duv, 2);
+      if (q == 0) {
+        s_dd[r][cl] = dd;
+        s_du[r][cl] = fmaf(Dc, ev, duv);
+        dDacc = fmaf(ev, uu, dDacc);
+      }
+      // sums over channels: the 8 channels of the warp by shuffles, then the block's warps by shared-memory atomics
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float vb = c_ok ? dBp[i] : 0.0f, vc = dCp[i];
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+          vb += __shfl_xor_sync(0xffffffffu, vb, o);
+          vc += __shfl_xor_sync(0xffffffffu, vc, o);
+        }
+        if (lane < 4) { atomicAdd(&s_dB[r][4 * q + i], vb); atomicAdd(&s_dC[r][4 * q + i], vc); }
+      }
+    }
+    __syncthreads();
+
+    // ---- write the chunk's outputs
+    for (int i = tid; i < CK * BCH; i += BT) {
+      const int r = i / BCH, j = i % BCH;
+      if (r < nt && c_base + j < p.De) {
+        const size_t e = (b * p.L + t0 + r) * p.De + c_base + j;
+        p.ddelta[e] = s_dd[r][j];
+        du[e] = from_f32<T>(s_du[r][j]);
+        if (z) {
+          const float zz = s_z[r][j], sg = sigmoid_f(zz);
+          dz[e] = from_f32<T>(s_dy[r][j] * s_y[r][j] * sg * (1.0f + zz * (1.0f - sg)));
+        }
+      }
+    }
+    for (int i = tid; i < CK * NST; i += BT) {
+      const int r = i / NST, n = i % NST;
+      if (r < nt) {
+        atomicAdd(p.dBm + (b * p.L + t0 + r) * NST + n, s_dB[r][n]);
+        atomicAdd(p.dCm + (b * p.L + t0 + r) * NST + n, s_dC[r][n]);
+      }
+    }
+    __syncthreads();
+  }
+
+  if (c_ok) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      atomicAdd(p.dA + (size_t)c * NST + 4 * q + i, dAacc[i]);
+      if (p.dh0) p.dh0[(b * p.De + c) * NST + 4 * q + i] = g[i];
+    }
+    if (q == 0 && p.dD) atomicAdd(p.dD + c, dDacc);
+  }
+}
+
+}  // namespace
+
+size_t scan_bwd_ws_bytes(int B, int De, int L) {
+  const size_t nck = (size_t)(L + CK - 1) / CK;
+  return align_up(sizeof(float) * (size_t)B * nck * De * NST, 256);
+}
+
+cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void* u, const float* delta, const float* A,
+                                 const float* Bm, const float* Cm, const float* D, const void* z, const float* h0,
+                                 const float* dh_last, void* du, float* ddelta, float* dA, float* dBm, float* dCm, float* dD,
+                                 void* dz, float* dh0, float* ckpt, cudaStream_t st) {
+  const int nck = (c.L + CK - 1) / CK;
+  const BwdArgs a{dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0, ckpt, c.L, c.d_inner, nck};
+  cudaError_t e = cudaMemsetAsync(dA, 0, sizeof(float) * (size_t)c.d_inner * NST, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(dBm, 0, sizeof(float) * (size_t)c.B * c.L * NST, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(dCm, 0, sizeof(float) * (size_t)c.B * c.L * NST, st);
+  if (e == cudaSuccess && dD) e = cudaMemsetAsync(dD, 0, sizeof(float) * (size_t)c.d_inner, st);
+  if (e != cudaSuccess) return e;
+  const dim3 grid((c.d_inner + BCH - 1) / BCH, c.B);
+  const bool zoh = c.disc_mode == 0, bf = c.dtype == ROM_BF16;
+  if (bf) {
+    if (zoh) scan_ckpt_kernel<__nv_bfloat16, true><<<grid, BT, 0, st>>>(a); else scan_ckpt_kernel<__nv_bfloat16, false><<<grid, BT, 0, st>>>(a);
+  } else {
+    if (zoh) scan_ckpt_kernel<float, true><<<grid, BT, 0, st>>>(a); else scan_ckpt_kernel<float, false><<<grid, BT, 0, st>>>(a);
+  }
+  count_launch();
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  auto kern = bf ? (zoh ? scan_bwd_kernel<__nv_bfloat16, true> : scan_bwd_kernel<__nv_bfloat16, false>)
+                 : (zoh ? scan_bwd_kernel<float, true> : scan_bwd_kernel<float, false>);
+  if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BWD_SMEM)) != cudaSuccess) return e;
+  kern<<<grid, BT, BWD_SMEM, st>>>(a);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace rom

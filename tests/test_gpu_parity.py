@@ -418,3 +418,71 @@ def test_argument_errors_launch_nothing():
     small_ws = g.ws[:1024]
     assert rb.rom_layer_forward(g.cfg, g.weights, g.dev["x"], g.out, None, None, None, small_ws, check=False) == -3
     g.forward()                                       # nothing was enqueued by the rejected calls; the layer still runs
+
+
+# ---------------------------------------------------------------------------------------------- debug checks, device-side timeout
+def _status_detail(ws):
+    v = ws[:12].view(torch.int32).cpu()
+    return int(v[0]), int(v[1]), int(v[2])
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(E=8, K=1, B=3, L=130), dict(E=6, K=2, router_bias_scale=4.0, L=513)])
+def test_debug_checks_pass_on_good_runs_and_change_nothing(kw):
+    s = small_shape(**kw)
+    p = synth.make_inputs(s, recipe="unit")
+    plain = GpuLayer(s, p)
+    want = plain.forward().clone()
+    g = GpuLayer(s, p, flags=rb.ROM_FLAG_DEBUG_CHECKS)
+    assert rb.workspace_size(g.cfg) > rb.workspace_size(plain.cfg)      # canaries between the sub-buffers
+    got = g.forward()                                                     # asserts a clean status word
+    assert torch.equal(got, want)
+    n_debug = rb.last_launch_count()
+    plain.forward()
+    assert n_debug == rb.last_launch_count() + 3                          # canary write, table check, canary compare
+
+
+def test_debug_checks_report_a_damaged_table_and_a_damaged_canary():
+    """The damage is planted from the host into the workspace of a finished forward; the checks run again on demand."""
+    s = small_shape(E=4, K=2, L=200)
+    p = synth.make_inputs(s, recipe="unit")
+    g = GpuLayer(s, p, flags=rb.ROM_FLAG_DEBUG_CHECKS)
+    g.forward()
+    roa = g.tap("row_of_assign", torch.int32, 1).view(-1)
+    saved = roa[5].clone()
+    roa[5] = 10 ** 6                                                      # a row far outside the padded range
+    rb.rom_debug_check(g.cfg, g.ws)
+    torch.cuda.synchronize()
+    assert _status_detail(g.ws) == (-8, 10, 5)
+    assert rb.rom_get_status(g.ws) == -8 and "debug check" in rb.status_string(-8)
+    roa[5] = saved
+    rb.rom_debug_check(g.cfg, g.ws)
+    assert rb.rom_get_status(g.ws) == 0
+    off, n = rb.workspace_find(g.cfg, "U")
+    canary = (off + n + 255) // 256 * 256                                 # the canary that follows U
+    g.ws[canary + 17] ^= 0xFF
+    rb.rom_debug_check(g.cfg, g.ws)
+    torch.cuda.synchronize()
+    code, where, _ = _status_detail(g.ws)
+    assert (code, where) == (-8, 20)
+    assert rb.rom_get_status(g.ws) == -8
+    g.forward()                                                           # canaries are rewritten by the next forward: clean again
+
+
+def test_device_wait_that_runs_out_is_reported_and_the_workspace_stays_usable():
+    """Fault injection on the host's request (ROM_FLAG_TEST_STALL): the producer of the first grouped projection never
+    issues the copies of one operand stage, so the MMA issuer's bounded wait runs out; the kernel must latch
+    ROM_ERR_DEVICE_TIMEOUT, wait for what it already issued, free its tensor memory and return; the launches after it
+    still run (on unspecified data, with valid indices).  The next ordinary forward on the same workspace is checked
+    against the oracle."""
+    s = small_shape(E=4, K=1, B=2, L=300, d_model=256)
+    p = synth.make_inputs(s, recipe="unit")
+    g = GpuLayer(s, p, flags=rb.ROM_FLAG_TEST_STALL)
+    rb.rom_layer_forward(g.cfg, g.weights, g.dev["x"], g.out, g.idx, g.gates, g.counts, g.ws)
+    torch.cuda.synchronize()
+    assert rb.rom_get_status(g.ws) == -6
+    good = GpuLayer(s, p)
+    good.ws = g.ws                                                        # same workspace, ordinary flags
+    out = good.forward()
+    ref, im = oracle_layer(s, p)
+    np.testing.assert_array_equal(good.idx.cpu().numpy(), im["idx"])
+    assert_close(np64(out), ref, TOL["bf16"], "out after a timed-out call")
