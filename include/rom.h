@@ -145,16 +145,14 @@ ROM_API int rom_route_balance(const rom_config *cfg, const void *x, const void *
  *
  * The caller passes inputs and outputs only; arguments, outputs and their meaning are those of
  * rom_route.  Limits: B*L <= 65536 tokens and B*L*K <= 131072 assignments (E <= 64, K <= 8 as
- * elsewhere), and the routing tables plus the fp64 copy of the router weights (8 * d_model * E bytes,
- * E rounded up to 8) must fit the 3 MiB; anything larger returns ROM_ERR_STATIC_SCRATCH and launches
- * nothing -- use rom_route with a caller-owned workspace instead.  The call itself allocates nothing,
- * on the host or device.
+ * elsewhere); anything larger returns ROM_ERR_STATIC_SCRATCH and launches nothing -- use rom_route
+ * with a caller-owned workspace instead.  The call itself allocates nothing, on the host or device.
  *
  * The first call on each GPU looks up the array's device address (once per device, with that
  * device current); make that first call before starting any stream capture.
  * All calls on one GPU share the array, and it keeps the previous call's contents.  Each call
- * rewrites what it reads and clears, on `stream`, the one table that must start cleared, so
- * back-to-back calls on one stream are safe; calls that overlap on the same GPU (other streams or
+ * rewrites what it reads, clears the one table that must start cleared and leaves its blocks-done
+ * counter at zero, so back-to-back calls on one stream are safe; calls that overlap on the same GPU (other streams or
  * host threads) race on the scratch and must be serialised by the caller.                          */
 ROM_API int rom_route_noalloc(const rom_config *cfg, const void *x, const void *W_r, const float *b_r,
                       int32_t *topk_idx, float *gates, int32_t *counts, int32_t *offsets,

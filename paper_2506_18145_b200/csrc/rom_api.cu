@@ -32,7 +32,6 @@ WsLayout make_layout(const rom_config& c) {
   l.num_m_tiles = take(sizeof(int32_t) * 4);
   l.tile_expert = take(sizeof(int32_t) * l.max_m_tiles);
   l.chunk_counts = take(sizeof(int32_t) * l.n_chunks * c.E);
-  l.wr_f64 = take(sizeof(double) * (size_t)c.d_model * ((c.E + 7) / 8 * 8));   // router weights in fp64, experts padded to 8
   l.chunk_prob = take(sizeof(double) * l.n_chunks * c.E);      // per-chunk softmax sums (rom_route_balance)
   l.topk_idx = take(sizeof(int32_t) * l.A);
   l.gates = take(sizeof(float) * l.A);
@@ -183,6 +182,7 @@ int rom_route(const rom_config* cfg, const void* x, const void* W_r, const float
   if ((rc = check_device()) != ROM_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   LaunchCounter::count = 0;
+  ROM_CUDA(cudaMemsetAsync(static_cast<char*>(ws) + lay.status, 0, sizeof(int32_t) * kStatusInts, st));
   ROM_CUDA(launch_route(*cfg, x, W_r, b_r, topk_idx, gates, counts, offsets, perm, inv_perm, static_cast<char*>(ws), lay, st));
   return ROM_OK;
 }
@@ -197,6 +197,7 @@ int rom_route_balance(const rom_config* cfg, const void* x, const void* W_r, con
   if (ws_bytes < lay.total) return ROM_ERR_WORKSPACE;
   if ((rc = check_device()) != ROM_OK) return rc;
   LaunchCounter::count = 0;
+  ROM_CUDA(cudaMemsetAsync(static_cast<char*>(ws) + lay.status, 0, sizeof(int32_t) * kStatusInts, static_cast<cudaStream_t>(stream)));
   ROM_CUDA(launch_balance(*cfg, x, W_r, b_r, alpha, F, Pbar, loss, static_cast<char*>(ws), lay, static_cast<cudaStream_t>(stream)));
   return ROM_OK;
 }
@@ -299,11 +300,11 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
   const bool debug_checks = (c.flags & ROM_FLAG_DEBUG_CHECKS) != 0;
   if (debug_checks) ROM_CUDA(launch_canaries(W, lay, false, st));
   // S1 + S2: router, top-K, permutation tables
-  ROM_CUDA(launch_route(c, x, w->W_r, w->b_r, topk_idx_out, gates, counts_out, nullptr, nullptr, nullptr, W, lay, st));
+  // ... and the token rows gathered into padded expert order (the second of the two launches copies them)
+  ROM_CUDA(launch_route_gather(c, x, w->W_r, w->b_r, topk_idx_out, gates, counts_out, W, lay, st));
   if (debug_checks) ROM_CUDA(launch_check_tables(c, W, lay, st));
   ROM_STAGE_DONE();
-  ROM_CUDA(launch_gather_rows(c, x, W, lay, st));
-  ROM_STAGE_DONE();
+  ROM_STAGE_DONE();      // "gather": fused into the routing launches
 
   auto gemm = [&](const void* A_, int lda, const void* B_, int ldb, int n_experts, int64_t bstride, int M_max, int Nn, int Kd,
                   const int32_t* te, const int32_t* nmt, const Epilogue& ep) -> cudaError_t {

@@ -19,6 +19,7 @@ constexpr int kStatusInts = 64;    // status block at the head of the workspace
 constexpr int kStatCode = 0;       // 0 or the rom_status a kernel latched (a wait that expired, an index out of range)
 constexpr int kStatWhere = 1;      // which wait gave up / which debug check failed (debug aid)
 constexpr int kStatIndex = 2;      // debug checks: the offending index
+constexpr int kStatTicket = 8;     // router: blocks-done counter (zero between calls)
 constexpr int kMaxCanaries = 40;   // sub-buffers of the workspace (debug checks put a canary after each)
 constexpr int kCanaryBytes = 256;
 
@@ -49,7 +50,7 @@ inline size_t scan_ws_floats(int B, int De, int L) {
 
 // Workspace carving, identical for every entry point (host arithmetic only).
 struct WsLayout {
-  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts, chunk_prob, wr_f64;
+  size_t status, counts, offsets, pad_offsets, num_m_tiles, tile_expert, chunk_counts, chunk_prob;
   size_t topk_idx, gates, perm, inv_perm, row_of_assign, assign_of_row;
   size_t x_perm, XZp, U, Zs, delta_r, Bm, Cm, Delta, Ygp, Op, scan_ws;
   size_t delta_rp, Bp, Cp, Dpre;      // per-expert x Proj / dt Proj only
@@ -106,10 +107,16 @@ cudaError_t launch_route(const rom_config& c, const void* x, const void* W_r, co
                          int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
                          int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, cudaStream_t st);
 
-// launch_route with the per-chunk sums of the router softmax as an extra output (chunk_prob [n_chunks, E] fp64, or nullptr).
+// launch_route with the per-chunk sums of the router softmax as an extra output (chunk_prob [n_chunks, E] fp64, or nullptr);
+// gather_x: also fill x_perm (the token rows in padded expert order, zero rows in the padding).
+// The status block of the workspace (its blocks-done counter) must be zero on entry; it is left zero.
 cudaError_t launch_route_stats(const rom_config& c, const void* x, const void* W_r, const float* b_r,
                                int32_t* topk_idx, float* gates, int32_t* counts, int32_t* offsets,
-                               int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, double* chunk_prob, cudaStream_t st);
+                               int32_t* perm, int32_t* inv_perm, char* ws, const WsLayout& lay, double* chunk_prob, cudaStream_t st,
+                               bool gather_x);
+// Router + tables + x_perm in two launches (the layer's path).
+cudaError_t launch_route_gather(const rom_config& c, const void* x, const void* W_r, const float* b_r,
+                                int32_t* topk_idx, float* gates, int32_t* counts, char* ws, const WsLayout& lay, cudaStream_t st);
 // Router + load-balance statistic: F[E], Pbar[E], loss[1] (device fp32, each may be null).
 cudaError_t launch_balance(const rom_config& c, const void* x, const void* W_r, const float* b_r, float alpha,
                            float* F, float* Pbar, float* loss, char* ws, const WsLayout& lay, cudaStream_t st);

@@ -34,13 +34,13 @@ WsLayout make_route_only_layout(const rom_config& c) {
   l.n_chunks = (l.T + kChunkTokens - 1) / kChunkTokens;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  l.status = take(sizeof(int32_t) * kStatusInts);      // only its blocks-done counter is used: zero at load, left zero by every call
   l.counts = take(sizeof(int32_t) * c.E);
   l.offsets = take(sizeof(int32_t) * (c.E + 1));
   l.pad_offsets = take(sizeof(int32_t) * (c.E + 1));
   l.num_m_tiles = take(sizeof(int32_t) * 4);
   l.tile_expert = take(sizeof(int32_t) * l.max_m_tiles);
   l.chunk_counts = take(sizeof(int32_t) * l.n_chunks * c.E);
-  l.wr_f64 = take(sizeof(double) * (size_t)c.d_model * ((c.E + 7) / 8 * 8));   // router weights in fp64, experts padded to 8
   l.topk_idx = take(sizeof(int32_t) * l.A);
   l.row_of_assign = take(sizeof(int32_t) * l.A);
   l.assign_of_row = take(sizeof(int32_t) * l.rows_max);

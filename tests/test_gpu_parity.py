@@ -169,7 +169,7 @@ def check_layer(s, recipe, with_D=True, gate_mode=0, disc_mode=0, flags=0, check
         rows = g.tap("row_of_assign", torch.int32, 1).view(-1)[::s.K].long()      # slot 0 row of each token
         assert_close(np64(g.tap("Ygp", tdt, s.d_inner)[rows]), im["Yg"], tol, "Yg")
     e = assert_close(np64(out), ref, tol, "out")
-    assert rb.last_launch_count() >= 9
+    assert rb.last_launch_count() >= 6
     return e
 
 
