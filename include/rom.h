@@ -206,6 +206,39 @@ ROM_API int rom_layer_forward(const rom_config *cfg, const rom_weights *w, const
                       int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
                       void *ws, size_t ws_bytes, void *stream);
 
+/* Backward pass of one RoM layer (Section 5.1: the layer is trained end to end; Appendix A.3: the router is trained
+ * through the gate values).  Given dout = dLoss/dO for the forward of rom_layer_forward on the same cfg, weights and
+ * x, returns dx = dLoss/dX and the gradient of every weight.  The equations reversed are those of Sections 3.1 and
+ * 4.2 as listed at rom_layer_forward.  Readings where the paper is silent: the top-K indicator is piecewise constant
+ * and is held fixed, so the router receives gradient only through R_i (gate_mode decides which form), not through the
+ * Conv/Gate projections, which carry the indicator alone; jitter noise and SparseMixer (Appendix A.3) are stochastic
+ * training-time estimators and are not part of this call.  Only the shared x Proj / dt Proj wiring (Section 4.3) is
+ * differentiated: cfg->small_proj_experts == E returns ROM_ERR_UNSUPPORTED.
+ * The call recomputes the forward activations it needs from x (it does not read a forward workspace), then walks the
+ * steps backwards: data gradients of the projections are the forward grouped GEMMs on transposed weights; weight
+ * gradients are sums over the tokens of each expert's segment.
+ *   x, dout, dx : [B, L, d_model] dtype.
+ *   g           : device pointers, fp32, fully overwritten: the shapes of the corresponding rom_weights fields;
+ *                 db_r may be NULL (not produced); dD is NULL exactly when w->D is.
+ *   ws          : rom_layer_backward_workspace_size(cfg) bytes.
+ * Sums that cross thread blocks use floating-point atomics: the last bits of the gradients vary from run to run.  */
+typedef struct {
+  float *dW_r;      /* [E, d_model]                    */
+  float *db_r;      /* [E] or NULL                     */
+  float *dW_inz;    /* [E, 2*d_inner, d_model]         */
+  float *dw_conv;   /* [d_conv, d_inner]               */
+  float *db_conv;   /* [d_inner]                       */
+  float *dW_x;      /* [dt_rank+2*d_state, d_inner]    */
+  float *dW_dt;     /* [d_inner, dt_rank]              */
+  float *db_dt;     /* [d_inner]                       */
+  float *dA;        /* [d_inner, d_state]              */
+  float *dD;        /* [d_inner] or NULL               */
+  float *dW_out;    /* [E, d_model, d_inner]           */
+} rom_grads;
+ROM_API int rom_layer_backward_workspace_size(const rom_config *cfg, size_t *bytes);
+ROM_API int rom_layer_backward(const rom_config *cfg, const rom_weights *w, const void *x, const void *dout, void *dx,
+                       const rom_grads *g, void *ws, size_t ws_bytes, void *stream);
+
 /* rom_layer_forward with HOST input and output: enqueues on `stream` the copy of x_host to x_dev, the
  * forward (x_dev -> out_dev) and the copy of out_dev to out_host, and returns without waiting.
  *   x_host, out_host : HOST pointers, [B, L, d_model] dtype; page-locked memory makes the copies

@@ -25,7 +25,8 @@ EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "
            "rom_get_status", "rom_status_string", "rom_last_launch_count", "rom_layer_forward_profile",
            "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance",
            "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step", "rom_layer_forward_host",
-           "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward")
+           "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward",
+           "rom_layer_backward_workspace_size", "rom_layer_backward")
 
 
 class RomConfig(ctypes.Structure):
@@ -37,6 +38,11 @@ class RomConfig(ctypes.Structure):
 class RomWeights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("W_r", "b_r", "W_inz", "w_conv", "b_conv", "W_x", "W_dt", "b_dt", "A", "D", "W_out")]
+
+
+class RomGrads(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("dW_r", "db_r", "dW_inz", "dw_conv", "db_conv", "dW_x", "dW_dt", "db_dt", "dA", "dD", "dW_out")]
 
 
 class RomError(RuntimeError):
@@ -62,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.rom_scan_workspace_size.argtypes = [cfgp, szp]
         L.rom_debug_check.argtypes = [cfgp, vp, ctypes.c_size_t, vp]
         L.rom_scan_backward_workspace_size.argtypes = [cfgp, szp]
+        L.rom_layer_backward_workspace_size.argtypes = [cfgp, szp]
+        L.rom_layer_backward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, vp, ctypes.POINTER(RomGrads), vp, ctypes.c_size_t, vp]
         L.rom_scan_backward.argtypes = [cfgp] + [vp] * 19 + [ctypes.c_size_t, vp]
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
         L.rom_route_noalloc.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
@@ -131,7 +139,8 @@ def scan_workspace_size(cfg: RomConfig) -> int:
     n = ctypes.c_size_t(0)
     rc = lib().rom_scan_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
     if rc != ROM_OK:
-        raise RomError(rc, "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward")
+        raise RomError(rc, "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward",
+           "rom_layer_backward_workspace_size", "rom_layer_backward")
     return int(n.value)
 
 
@@ -196,6 +205,26 @@ def rom_scan_backward(cfg, dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelt
                                  _ptr(dz), _ptr(dh0), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_scan_backward")
+    return rc
+
+
+def layer_backward_workspace_size(cfg: RomConfig) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().rom_layer_backward_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_layer_backward_workspace_size")
+    return int(n.value)
+
+
+def make_grads(g: Dict[str, Optional[torch.Tensor]]) -> RomGrads:
+    return RomGrads(*[_ptr(g.get(n)) for n, _ in RomGrads._fields_])
+
+
+def rom_layer_backward(cfg, weights: RomWeights, x, dout, dx, grads: RomGrads, ws, stream=None, check=True) -> int:
+    rc = lib().rom_layer_backward(ctypes.byref(cfg), ctypes.byref(weights), _ptr(x), _ptr(dout), _ptr(dx), ctypes.byref(grads), _ptr(ws),
+                                  ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_layer_backward")
     return rc
 
 

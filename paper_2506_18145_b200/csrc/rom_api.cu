@@ -247,7 +247,7 @@ int rom_scan_backward(const rom_config* cfg, const void* dy, const void* u, cons
   if ((rc = check_device()) != ROM_OK) return rc;
   LaunchCounter::count = 0;
   ROM_CUDA(launch_scan_backward(*cfg, dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0,
-                                static_cast<float*>(ws), static_cast<cudaStream_t>(stream)));
+                                static_cast<float*>(ws), cfg->d_inner, static_cast<cudaStream_t>(stream)));
   return ROM_OK;
 }
 
@@ -399,7 +399,167 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
 }  // namespace
 }  // namespace rom
 
+namespace rom {
+namespace {
+
+// Scratch of rom_layer_backward: the forward workspace (routing tables and recomputed activations) followed by the
+// gradient buffers and the transposed weights.
+struct BwdLayout {
+  size_t HZs, D32, dOp, dYgu, dYg, rowscale, dgate, dU1, ddelta, dBm, dCm, dpre, dxdbl, dU2, dHZs, dHZp, dxp, dlogit;
+  size_t WoT, WiT, WdtT, WxT, ckpt, total;
+};
+BwdLayout make_bwd_layout(const rom_config& c, const WsLayout& l) {
+  BwdLayout b{};
+  size_t o = align_up(l.total, 256);
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  const size_t T = (size_t)l.T, rows = (size_t)l.rows_max, De = c.d_inner, Dm = c.d_model, N = c.d_state, R = c.dt_rank, esz = l.esz;
+  b.HZs = take(esz * T * 2 * De);
+  b.D32 = take(4 * T * De);
+  b.dOp = take(esz * rows * Dm);
+  b.dYgu = take(esz * rows * De);
+  b.dYg = take(esz * T * De);
+  b.rowscale = take(4 * rows);
+  b.dgate = take(4 * T * c.K);
+  b.dU1 = take(esz * T * De);
+  b.ddelta = take(4 * T * De);
+  b.dBm = take(4 * T * N);
+  b.dCm = take(4 * T * N);
+  b.dpre = take(esz * T * De);
+  b.dxdbl = take(esz * T * (R + 2 * N));
+  b.dU2 = take(esz * T * De);
+  b.dHZs = take(esz * T * 2 * De);
+  b.dHZp = take(esz * rows * 2 * De);
+  b.dxp = take(esz * rows * Dm);
+  b.dlogit = take(4 * T * c.E);
+  b.WoT = take(esz * (size_t)c.E * De * Dm);
+  b.WiT = take(esz * (size_t)c.E * Dm * 2 * De);
+  b.WdtT = take(esz * R * De);
+  b.WxT = take(esz * De * (R + 2 * N));
+  b.ckpt = take(scan_bwd_ws_bytes(c.B, c.d_inner, c.L));
+  b.total = o;
+  return b;
+}
+
+}  // namespace
+}  // namespace rom
+
 extern "C" {
+
+int rom_layer_backward_workspace_size(const rom_config* cfg, size_t* bytes) {
+  if (!bytes) return ROM_ERR_INVALID_ARG;
+  const int rc = check_config(cfg, 0);
+  if (rc != ROM_OK) return rc;
+  *bytes = make_bwd_layout(*cfg, make_layout(*cfg)).total;
+  return ROM_OK;
+}
+
+int rom_layer_backward(const rom_config* cfg, const rom_weights* w, const void* x, const void* dout, void* dx, const rom_grads* g,
+                       void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg, 0);
+  if (rc != ROM_OK) return rc;
+  if (cfg->small_proj_experts > 1) return ROM_ERR_UNSUPPORTED;      // only the shared x Proj / dt Proj wiring is differentiated
+  if (!w || !x || !dout || !dx || !g || !ws) return ROM_ERR_INVALID_ARG;
+  if (!w->W_r || !w->W_inz || !w->w_conv || !w->W_x || !w->W_dt || !w->A || !w->W_out) return ROM_ERR_INVALID_ARG;
+  if (!g->dW_r || !g->dW_inz || !g->dw_conv || !g->db_conv || !g->dW_x || !g->dW_dt || !g->db_dt || !g->dA || !g->dW_out) return ROM_ERR_INVALID_ARG;
+  if ((w->D == nullptr) != (g->dD == nullptr)) return ROM_ERR_INVALID_ARG;
+  const void* ptrs[] = {x, dout, dx, ws, w->W_r, w->W_inz, w->w_conv, w->W_x, w->W_dt, w->A, w->W_out, g->dW_r, g->dW_inz, g->dw_conv,
+                        g->db_conv, g->dW_x, g->dW_dt, g->db_dt, g->dA, g->dW_out};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return ROM_ERR_INVALID_ARG;
+  const rom_config& c = *cfg;
+  const WsLayout lay = make_layout(c);
+  const BwdLayout bl = make_bwd_layout(c, lay);
+  if (ws_bytes < bl.total) return ROM_ERR_WORKSPACE;
+  if ((rc = check_device()) != ROM_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* W = static_cast<char*>(ws);
+  LaunchCounter::count = 0;
+
+  const int T = (int)lay.T, De = c.d_inner, Dm = c.d_model, R = c.dt_rank, N = c.d_state, rows = (int)lay.rows_max;
+  const size_t esz = lay.esz;
+  const bool tc = c.dtype == ROM_BF16 && !(c.flags & ROM_FLAG_SIMT_GEMM);
+  int32_t* status = reinterpret_cast<int32_t*>(W + lay.status);
+  const int32_t* tile_expert = reinterpret_cast<int32_t*>(W + lay.tile_expert);
+  const int32_t* num_m_tiles = reinterpret_cast<int32_t*>(W + lay.num_m_tiles);
+  const int32_t* row_of_assign = reinterpret_cast<int32_t*>(W + lay.row_of_assign);
+  const int32_t* pad_offsets = reinterpret_cast<int32_t*>(W + lay.pad_offsets);
+  float* gates = reinterpret_cast<float*>(W + lay.gates);
+  float* Bm = reinterpret_cast<float*>(W + lay.Bm);
+  float* Cm = reinterpret_cast<float*>(W + lay.Cm);
+  auto gemm = [&](const void* A_, int lda, const void* B_, int ldb, int n_experts, int64_t bstride, int M_max, int Nn, int Kd,
+                  const int32_t* te, const int32_t* nmt, const Epilogue& ep) -> cudaError_t {
+    if (tc) return launch_gemm_tc(A_, lda, B_, ldb, n_experts, M_max, Nn, Kd, te, nmt, ep, status, st);
+    return launch_gemm_simt(c.dtype, A_, lda, B_, ldb, bstride, M_max, Nn, Kd, te, nmt, ep, st);
+  };
+  auto store_to = [&](void* C_, int ldc) { return Epilogue{EPI_STORE, C_, ldc, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr}; };
+
+  // ---- forward, recomputed with the raw Gate Proj rows kept (the forward proper stores them activated at top-1)
+  ROM_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t) * kStatusInts, st));
+  ROM_CUDA(launch_route_gather(c, x, w->W_r, w->b_r, nullptr, gates, nullptr, W, lay, st));
+  ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, rows, 2 * De, Dm, tile_expert, num_m_tiles, store_to(W + lay.XZp, 2 * De)));
+  ROM_CUDA(launch_slot_sum(c.dtype, W + lay.XZp, row_of_assign, W + bl.HZs, T, 2 * De, c.K, st));       // H_t, Z_t: sums over the selected experts
+  rom_config c1 = c;
+  c1.K = 1;
+  ROM_CUDA(launch_conv(c1, W + bl.HZs, nullptr, w->w_conv, w->b_conv, W + lay.U, nullptr, st));
+  Epilogue e_x{EPI_XPROJ, W + lay.delta_r, R, Bm, Cm, nullptr, R, N, nullptr, nullptr};
+  ROM_CUDA(gemm(W + lay.U, De, w->W_x, De, 1, 0, T, R + 2 * N, De, nullptr, nullptr, e_x));
+  Epilogue e_dt{EPI_SOFTPLUS, W + lay.Delta, De, nullptr, nullptr, w->b_dt, 0, 0, nullptr, nullptr};
+  ROM_CUDA(gemm(W + lay.delta_r, R, w->W_dt, R, 1, 0, T, De, R, nullptr, nullptr, e_dt));
+  float* D32 = reinterpret_cast<float*>(W + bl.D32);
+  ROM_CUDA(launch_cast_f32(c.dtype, W + lay.Delta, D32, (long long)T * De, st));
+  // gated scan output in expert order (operand of the Out Proj weight gradient); padding rows must be zero
+  ROM_CUDA(cudaMemsetAsync(W + lay.Ygp, 0, esz * (size_t)rows * De, st));
+  const char* zraw = W + bl.HZs + (size_t)De * esz;
+  ROM_CUDA(launch_scan(c, W + lay.U, W + lay.Delta, false, w->A, Bm, Cm, w->D, zraw, 2 * De, nullptr, nullptr, W + lay.Ygp, nullptr,
+                       row_of_assign, c.K, reinterpret_cast<float*>(W + lay.scan_ws), false, st));
+
+  // ---- Out Proj and combine, reversed: back_k = dO_t W_out,k; dYg, dgate; dW_out
+  ROM_CUDA(launch_gather_rows_to(c, dout, W + bl.dOp, Dm, W, lay, st));
+  ROM_CUDA(launch_transpose(c.dtype, w->W_out, W + bl.WoT, c.E, Dm, De, st));
+  ROM_CUDA(gemm(W + bl.dOp, Dm, W + bl.WoT, Dm, c.E, (int64_t)De * Dm, rows, De, Dm, tile_expert, num_m_tiles, store_to(W + bl.dYgu, De)));
+  float* rowscale = reinterpret_cast<float*>(W + bl.rowscale);
+  float* dgate = reinterpret_cast<float*>(W + bl.dgate);
+  ROM_CUDA(cudaMemsetAsync(rowscale, 0, sizeof(float) * rows, st));
+  ROM_CUDA(launch_combine_bwd(c.dtype, W + bl.dYgu, W + lay.Ygp, row_of_assign, gates, W + bl.dYg, dgate, rowscale, T, De, c.K, st));
+  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dOp, Dm, W + lay.Ygp, De, rowscale, pad_offsets, c.E, rows, Dm, De, g->dW_out, st));
+
+  // ---- gate and scan, reversed
+  float* ddelta = reinterpret_cast<float*>(W + bl.ddelta);
+  float* dBm = reinterpret_cast<float*>(W + bl.dBm);
+  float* dCm = reinterpret_cast<float*>(W + bl.dCm);
+  ROM_CUDA(launch_scan_backward(c, W + bl.dYg, W + lay.U, D32, w->A, Bm, Cm, w->D, zraw, nullptr, nullptr, W + bl.dU1, ddelta, g->dA, dBm, dCm,
+                                g->dD, W + bl.dHZs + (size_t)De * esz, nullptr, reinterpret_cast<float*>(W + bl.ckpt), 2 * De, st));
+
+  // ---- dt Proj and x Proj, reversed
+  ROM_CUDA(cudaMemsetAsync(g->db_dt, 0, sizeof(float) * De, st));
+  ROM_CUDA(launch_softplus_bwd(c.dtype, ddelta, D32, W + bl.dpre, g->db_dt, T, De, st));
+  ROM_CUDA(launch_transpose(c.dtype, w->W_dt, W + bl.WdtT, 1, De, R, st));
+  ROM_CUDA(gemm(W + bl.dpre, De, W + bl.WdtT, De, 1, 0, T, R, De, nullptr, nullptr, store_to(W + bl.dxdbl, R + 2 * N)));      // d(delta) into columns [0, R)
+  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dpre, De, W + lay.delta_r, R, nullptr, nullptr, 1, T, De, R, g->dW_dt, st));
+  ROM_CUDA(launch_pack_bc(c.dtype, dBm, dCm, W + bl.dxdbl, T, R, N, st));
+  ROM_CUDA(launch_transpose(c.dtype, w->W_x, W + bl.WxT, 1, R + 2 * N, De, st));
+  ROM_CUDA(gemm(W + bl.dxdbl, R + 2 * N, W + bl.WxT, R + 2 * N, 1, 0, T, De, R + 2 * N, nullptr, nullptr, store_to(W + bl.dU2, De)));
+  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dxdbl, R + 2 * N, W + lay.U, De, nullptr, nullptr, 1, T, R + 2 * N, De, g->dW_x, st));
+
+  // ---- conv, reversed (dU = scan part + x Proj part)
+  ROM_CUDA(cudaMemsetAsync(g->dw_conv, 0, sizeof(float) * (size_t)c.d_conv * De, st));
+  ROM_CUDA(cudaMemsetAsync(g->db_conv, 0, sizeof(float) * De, st));
+  ROM_CUDA(launch_conv_bwd(c, W + bl.HZs, w->w_conv, w->b_conv, W + bl.dU1, W + bl.dU2, W + bl.dHZs, g->dw_conv, g->db_conv, st));
+
+  // ---- Conv Proj | Gate Proj, reversed: every selected expert of a token receives the token's (dH, dZ)
+  ROM_CUDA(launch_gather_rows_to(c, W + bl.dHZs, W + bl.dHZp, 2 * De, W, lay, st));
+  ROM_CUDA(launch_transpose(c.dtype, w->W_inz, W + bl.WiT, c.E, 2 * De, Dm, st));
+  ROM_CUDA(gemm(W + bl.dHZp, 2 * De, W + bl.WiT, 2 * De, c.E, (int64_t)Dm * 2 * De, rows, Dm, 2 * De, tile_expert, num_m_tiles, store_to(W + bl.dxp, Dm)));
+  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dHZp, 2 * De, W + lay.x_perm, Dm, nullptr, pad_offsets, c.E, rows, 2 * De, Dm, g->dW_inz, st));
+
+  // ---- router, reversed (through the gate values only), and dx
+  float* dlogit = reinterpret_cast<float*>(W + bl.dlogit);
+  ROM_CUDA(cudaMemsetAsync(g->dW_r, 0, sizeof(float) * (size_t)c.E * Dm, st));
+  if (g->db_r) ROM_CUDA(cudaMemsetAsync(g->db_r, 0, sizeof(float) * c.E, st));
+  ROM_CUDA(launch_router_bwd(c, x, w->W_r, w->b_r, reinterpret_cast<const int32_t*>(W + lay.topk_idx), gates, dgate, dlogit, g->db_r, g->dW_r, st));
+  ROM_CUDA(launch_dx(c, W + bl.dxp, row_of_assign, dlogit, w->W_r, dx, st));
+  return ROM_OK;
+}
 
 int rom_layer_forward(const rom_config* cfg, const rom_weights* w, const void* x, void* out, int32_t* topk_idx_out,
                       float* gates_out, int32_t* counts_out, void* ws, size_t ws_bytes, void* stream) {

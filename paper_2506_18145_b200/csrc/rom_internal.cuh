@@ -177,7 +177,26 @@ size_t scan_bwd_ws_bytes(int B, int De, int L);
 cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void* u, const float* delta, const float* A,
                                  const float* Bm, const float* Cm, const float* D, const void* z, const float* h0,
                                  const float* dh_last, void* du, float* ddelta, float* dA, float* dBm, float* dCm, float* dD,
-                                 void* dz, float* dh0, float* ckpt, cudaStream_t st);
+                                 void* dz, float* dh0, float* ckpt, int ldz /* row pitch of z and dz */, cudaStream_t st);
+
+// Pieces of the layer's backward pass (rom_backward.cu); dtype tensors per the config, sums in fp32.
+cudaError_t launch_transpose(int dtype, const void* in, void* out, int batch, int R, int C, cudaStream_t st);      // out[b][c][r] = in[b][r][c]
+cudaError_t launch_slot_sum(int dtype, const void* src, const int32_t* row_of_assign, void* dst, long long Tn, int width, int K, cudaStream_t st);
+cudaError_t launch_cast_f32(int dtype, const void* in, float* out, long long n, cudaStream_t st);
+cudaError_t launch_combine_bwd(int dtype, const void* dYgu, const void* Ygp, const int32_t* row_of_assign, const float* gates, void* dYg,
+                               float* dgate, float* rowscale, long long Tn, int De, int K, cudaStream_t st);
+cudaError_t launch_softplus_bwd(int dtype, const float* ddelta, const float* Delta32, void* dpre, float* db_dt, long long Tn, int De, cudaStream_t st);
+cudaError_t launch_pack_bc(int dtype, const float* dBm, const float* dCm, void* dxdbl, long long Tn, int R, int N, cudaStream_t st);
+cudaError_t launch_conv_bwd(const rom_config& c, const void* HZ, const void* w_conv, const float* b_conv, const void* dU1, const void* dU2,
+                            void* dHZ, float* dw, float* db, cudaStream_t st);
+cudaError_t launch_router_bwd(const rom_config& c, const void* x, const void* W_r, const float* b_r, const int32_t* idx, const float* gates,
+                              const float* dgate, float* dlogit, float* db_r, float* dW_r, cudaStream_t st);
+cudaError_t launch_dx(const rom_config& c, const void* dxp, const int32_t* row_of_assign, const float* dlogit, const void* W_r, void* dx,
+                      cudaStream_t st);
+// C[s][P, Q] = sum over rows r of segment s of scale[r] X[r, :P]^T Y[r, :Q]; seg: n_seg + 1 row offsets (device) or nullptr = one
+// segment of rows_total rows; scale may be nullptr.
+cudaError_t launch_wgrad(int dtype, const void* X, int ldx, const void* Y, int ldy, const float* scale, const int32_t* seg, int n_seg,
+                         int rows_total, int P, int Q, float* C, cudaStream_t st);
 
 cudaError_t launch_combine(const rom_config& c, const void* Op, const int32_t* row_of_assign, const float* gates,
                            void* out, cudaStream_t st);

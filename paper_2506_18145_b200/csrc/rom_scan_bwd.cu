@@ -31,6 +31,7 @@ struct BwdArgs {
   void* du; float* ddelta; float* dA; float* dBm; float* dCm; float* dD; void* dz; float* dh0;
   float* ckpt;        // [B, nck, De, 16]
   int L, De, nck;
+  int ldz;            // row pitch (elements) of z and dz
 };
 
 __device__ __forceinline__ float sigmoid_f(float v) { return 1.0f / (1.0f + expf(-v)); }
@@ -115,7 +116,7 @@ scan_bwd_kernel(const BwdArgs p) {
       if (r < nt && c_base + j < p.De) {
         const size_t e = (b * p.L + t0 + r) * p.De + c_base + j;
         dl = p.delta[e]; uu = to_f32(u[e]); dyv = to_f32(dy[e]);
-        if (z) zz = to_f32(z[e]);
+        if (z) zz = to_f32(z[(b * p.L + t0 + r) * p.ldz + c_base + j]);
       }
       s_dl[r][j] = dl; s_u[r][j] = uu; s_dy[r][j] = dyv; s_z[r][j] = zz;
       s_e[r][j] = z ? dyv * zz * sigmoid_f(zz) : dyv;
@@ -214,7 +215,7 @@ scan_bwd_kernel(const BwdArgs p) {
         du[e] = from_f32<T>(s_du[r][j]);
         if (z) {
           const float zz = s_z[r][j], sg = sigmoid_f(zz);
-          dz[e] = from_f32<T>(s_dy[r][j] * s_y[r][j] * sg * (1.0f + zz * (1.0f - sg)));
+          dz[(b * p.L + t0 + r) * p.ldz + c_base + j] = from_f32<T>(s_dy[r][j] * s_y[r][j] * sg * (1.0f + zz * (1.0f - sg)));
         }
       }
     }
@@ -248,9 +249,9 @@ size_t scan_bwd_ws_bytes(int B, int De, int L) {
 cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void* u, const float* delta, const float* A,
                                  const float* Bm, const float* Cm, const float* D, const void* z, const float* h0,
                                  const float* dh_last, void* du, float* ddelta, float* dA, float* dBm, float* dCm, float* dD,
-                                 void* dz, float* dh0, float* ckpt, cudaStream_t st) {
+                                 void* dz, float* dh0, float* ckpt, int ldz, cudaStream_t st) {
   const int nck = (c.L + CK - 1) / CK;
-  const BwdArgs a{dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0, ckpt, c.L, c.d_inner, nck};
+  const BwdArgs a{dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0, ckpt, c.L, c.d_inner, nck, ldz};
   cudaError_t e = cudaMemsetAsync(dA, 0, sizeof(float) * (size_t)c.d_inner * NST, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(dBm, 0, sizeof(float) * (size_t)c.B * c.L * NST, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(dCm, 0, sizeof(float) * (size_t)c.B * c.L * NST, st);

@@ -77,3 +77,65 @@ def test_scan_backward_argument_errors():
     bad = list(args); bad[6] = t                   # D without dD
     assert rb.rom_scan_backward(cfg, *bad, ws, check=False) == -1
     assert rb.rom_scan_backward(cfg, *args, ws[:64], check=False) == -3
+
+
+# ---------------------------------------------------------------------------------------------- the whole layer
+GRAD_NAMES = ("dW_r", "db_r", "dW_inz", "dw_conv", "db_conv", "dW_x", "dW_dt", "db_dt", "dA", "dD", "dW_out")
+
+
+def run_layer_backward(s, recipe="unit", gate_mode=0, disc_mode=0, flags=0, with_D=True, seed=4242):
+    p = synth.make_inputs(s, recipe=recipe, with_D=with_D)
+    tdt = synth.torch_dtype(s)
+    g = torch.Generator().manual_seed(seed)
+    dout = torch.randn(p["x"].shape, generator=g).to(tdt)
+    cfg = rb.config_from_shape(s, gate_mode, disc_mode, flags)
+    dev = {k: (None if v is None else v.cuda().contiguous()) for k, v in p.items()}
+    weights = rb.make_weights(dev)
+    grads = {n: torch.empty(p[n[1:]].shape, dtype=torch.float32, device="cuda") for n in GRAD_NAMES if p.get(n[1:]) is not None}
+    if "db_r" not in grads:                       # no router bias in the forward: its gradient is still defined, ask for it
+        grads["db_r"] = torch.empty((s.E,), dtype=torch.float32, device="cuda")
+    dx = torch.empty_like(dev["x"])
+    ws = torch.empty(rb.layer_backward_workspace_size(cfg), dtype=torch.uint8, device="cuda")
+    rb.rom_layer_backward(cfg, weights, dev["x"], dout.cuda(), dx, rb.make_grads(grads), ws)
+    torch.cuda.synchronize()
+    assert rb.rom_get_status(ws) == 0
+    f = lambda v: None if v is None else np64(v)
+    ref = G.rom_layer_backward(f(dout), f(p["x"]), f(p["W_r"]), f(p["b_r"]), f(p["W_inz"]), f(p["w_conv"]), f(p["b_conv"]), f(p["W_x"]),
+                               f(p["W_dt"]), f(p["b_dt"]), f(p["A"]), f(p["D"]), f(p["W_out"]), K=s.K, dt_rank=s.dt_rank,
+                               gate_mode=gate_mode, disc_mode=disc_mode)
+    tol = TOL[s.dtype]
+    assert_close(np64(dx), ref["dx"], tol, "dx")
+    for n, t in grads.items():
+        assert_close(np64(t), ref[n], tol, n)
+
+
+def bshape(**kw):
+    base = dict(name="b", B=2, L=150, d_model=128, d_inner=256, d_state=16, d_conv=4, dt_rank=16, E=4, K=2, dtype="bf16", seed_base=66000)
+    base.update(kw)
+    return synth.RomShape(**base)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),                                              # top-2, ragged L
+    dict(E=8, K=1, B=3, L=130),                          # top-1
+    dict(E=3, K=3, L=64, d_conv=3),
+    dict(E=6, K=2, router_bias_scale=2.0, L=257, d_conv=2, dt_rank=32),
+])
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", rb.ROM_FLAG_SIMT_GEMM), ("bf16", 0)])
+def test_layer_backward_parity(kw, dtype, flags):
+    run_layer_backward(bshape(dtype=dtype, **kw), flags=flags)
+
+
+@pytest.mark.parametrize("gate_mode,disc_mode", [(1, 0), (0, 1), (1, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_layer_backward_modes(gate_mode, disc_mode, dtype):
+    run_layer_backward(bshape(dtype=dtype, L=200), gate_mode=gate_mode, disc_mode=disc_mode)
+
+
+def test_layer_backward_without_skip_and_single_expert():
+    run_layer_backward(bshape(E=1, K=1, L=96, dtype="f32"), with_D=False)
+
+
+def test_layer_backward_small_bf16_config():
+    """The small bf16 configuration (B=4, L=2048, d_model=1024, d_inner=2048, 8 experts, top-1) on the tensor path."""
+    run_layer_backward(synth.CONFIGS["small_bf16"])
