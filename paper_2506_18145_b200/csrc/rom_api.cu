@@ -406,7 +406,7 @@ namespace {
 // gradient buffers and the transposed weights.
 struct BwdLayout {
   size_t HZs, D32, dOp, dYgu, dYg, rowscale, dgate, dU1, ddelta, dBm, dCm, dpre, dxdbl, dU2, dHZs, dHZp, dxp, dlogit;
-  size_t WoT, WiT, WdtT, WxT, ckpt, total;
+  size_t WoT, WiT, WdtT, WxT, ckpt, Xt, Yt, total;
 };
 BwdLayout make_bwd_layout(const rom_config& c, const WsLayout& l) {
   BwdLayout b{};
@@ -436,6 +436,10 @@ BwdLayout make_bwd_layout(const rom_config& c, const WsLayout& l) {
   b.WdtT = take(esz * R * De);
   b.WxT = take(esz * De * (R + 2 * N));
   b.ckpt = take(scan_bwd_ws_bytes(c.B, c.d_inner, c.L));
+  // tensor path: the activations of the two grouped weight gradients, transposed (token rows contiguous)
+  const bool tcw = c.dtype == ROM_BF16 && !(c.flags & ROM_FLAG_SIMT_GEMM);
+  b.Xt = take(tcw ? esz * 2 * De * rows : 0);
+  b.Yt = take(tcw ? esz * (De > Dm ? De : Dm) * rows : 0);
   b.total = o;
   return b;
 }
@@ -521,7 +525,16 @@ int rom_layer_backward(const rom_config* cfg, const rom_weights* w, const void* 
   float* dgate = reinterpret_cast<float*>(W + bl.dgate);
   ROM_CUDA(cudaMemsetAsync(rowscale, 0, sizeof(float) * rows, st));
   ROM_CUDA(launch_combine_bwd(c.dtype, W + bl.dYgu, W + lay.Ygp, row_of_assign, gates, W + bl.dYg, dgate, rowscale, T, De, c.K, st));
-  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dOp, Dm, W + lay.Ygp, De, rowscale, pad_offsets, c.E, rows, Dm, De, g->dW_out, st));
+  // grouped weight gradient (a sum over each expert's row segment): tensor path = the grouped GEMM over transposed
+  // activations with per-expert K ranges; otherwise the plain fp32-FMA kernel
+  auto grouped_wgrad = [&](const void* X, int P, const void* Y, int Q, const float* scale, float* C) -> cudaError_t {
+    if (!tc) return launch_wgrad(c.dtype, X, P, Y, Q, scale, pad_offsets, c.E, rows, P, Q, C, st);
+    cudaError_t e = launch_transpose_scaled(c.dtype, X, W + bl.Xt, rows, P, rows, scale, st);
+    if (e == cudaSuccess) e = launch_transpose_scaled(c.dtype, Y, W + bl.Yt, rows, Q, rows, nullptr, st);
+    if (e == cudaSuccess) e = launch_gemm_tc_wgrad(W + bl.Xt, W + bl.Yt, rows, pad_offsets, c.E, P, Q, C, status, st);
+    return e;
+  };
+  ROM_CUDA(grouped_wgrad(W + bl.dOp, Dm, W + lay.Ygp, De, rowscale, g->dW_out));
 
   // ---- gate and scan, reversed
   float* ddelta = reinterpret_cast<float*>(W + bl.ddelta);
@@ -550,7 +563,7 @@ int rom_layer_backward(const rom_config* cfg, const rom_weights* w, const void* 
   ROM_CUDA(launch_gather_rows_to(c, W + bl.dHZs, W + bl.dHZp, 2 * De, W, lay, st));
   ROM_CUDA(launch_transpose(c.dtype, w->W_inz, W + bl.WiT, c.E, 2 * De, Dm, st));
   ROM_CUDA(gemm(W + bl.dHZp, 2 * De, W + bl.WiT, 2 * De, c.E, (int64_t)Dm * 2 * De, rows, Dm, 2 * De, tile_expert, num_m_tiles, store_to(W + bl.dxp, Dm)));
-  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dHZp, 2 * De, W + lay.x_perm, Dm, nullptr, pad_offsets, c.E, rows, 2 * De, Dm, g->dW_inz, st));
+  ROM_CUDA(grouped_wgrad(W + bl.dHZp, 2 * De, W + lay.x_perm, Dm, nullptr, g->dW_inz));
 
   // ---- router, reversed (through the gate values only), and dx
   float* dlogit = reinterpret_cast<float*>(W + bl.dlogit);

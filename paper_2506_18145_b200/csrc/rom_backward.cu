@@ -50,6 +50,23 @@ transpose_kernel(const T* __restrict__ in, T* __restrict__ out, int R, int C) {
   }
 }
 
+// out[c][r] = scale[r] * in[r][c] (activations transposed for the tensor-core weight gradient; scale = the row's gate)
+template <typename T>
+__global__ void __launch_bounds__(256)
+transpose_scaled_kernel(const T* __restrict__ in, T* __restrict__ out, int R, int C, int ldo, const float* __restrict__ scale) {
+  __shared__ float tile[32][33];
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int r = r0 + i, c = c0 + threadIdx.x;
+    if (r < R && c < C) tile[i][threadIdx.x] = to_f32(in[(size_t)r * C + c]) * (scale ? scale[r] : 1.0f);
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += 8) {
+    const int c = c0 + i, r = r0 + threadIdx.x;
+    if (r < R && c < C) out[(size_t)c * ldo + r] = from_f32<T>(tile[threadIdx.x][i]);
+  }
+}
+
 // dst[t, :] = sum_k src[row_of_assign[t*K + k], :]  (ascending k, fp32 accumulation), rows `width` wide
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -353,6 +370,14 @@ cudaError_t launch_transpose(int dtype, const void* in, void* out, int batch, in
   const dim3 grid((C + 31) / 32, (R + 31) / 32, batch), block(32, 8);
   if (dtype == ROM_BF16) transpose_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)in, (__nv_bfloat16*)out, R, C);
   else transpose_kernel<float><<<grid, block, 0, st>>>((const float*)in, (float*)out, R, C);
+  count_launch();
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transpose_scaled(int dtype, const void* in, void* out, int R, int C, int ldo, const float* scale, cudaStream_t st) {
+  const dim3 grid((C + 31) / 32, (R + 31) / 32), block(32, 8);
+  if (dtype == ROM_BF16) transpose_scaled_kernel<__nv_bfloat16><<<grid, block, 0, st>>>((const __nv_bfloat16*)in, (__nv_bfloat16*)out, R, C, ldo, scale);
+  else transpose_scaled_kernel<float><<<grid, block, 0, st>>>((const float*)in, (float*)out, R, C, ldo, scale);
   count_launch();
   return cudaGetLastError();
 }

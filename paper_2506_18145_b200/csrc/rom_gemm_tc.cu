@@ -285,7 +285,8 @@ __global__ void __launch_bounds__(threads_of(MODE), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int M_max, int N, int Kd, int block_n, uint32_t idesc,
                const int32_t* __restrict__ tile_expert, const int32_t* __restrict__ num_m_tiles_dev,
-               Epilogue ep, int32_t* __restrict__ status, uint32_t wait_limit, int withhold_kb) {
+               Epilogue ep, int32_t* __restrict__ status, uint32_t wait_limit, int withhold_kb,
+               const int32_t* __restrict__ k_seg, int n_seg) {
   constexpr int STAGES = stages_of(MODE);
   constexpr int SB = stage_bytes_of(MODE);          // bytes per operand stage (multiple of 1024)
   extern __shared__ unsigned char smem_raw[];
@@ -309,8 +310,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const int M_valid = min(M_max, num_m_tiles * BLOCK_M);
   // EPI_SWIGLU: a tile holds 128 gate columns and the 128 up columns of the same hidden units
   const int n_tiles = MODE == EPI_SWIGLU ? N / 128 : (N + block_n - 1) / block_n;
-  const int total_tiles = num_m_tiles * n_tiles;
+  // Weight-gradient mode (k_seg != nullptr): n_seg independent problems share A and B; problem s contracts the K range
+  // [k_seg[s], k_seg[s+1]) (multiples of BLOCK_K; an expert's padded row segment) and writes rows [s M_max, (s+1) M_max) of C.
+  const int seg_tiles = num_m_tiles * n_tiles;
+  const int total_tiles = k_seg ? n_seg * seg_tiles : seg_tiles;
   const int num_kb = (Kd + BLOCK_K - 1) / BLOCK_K;
+  auto decode = [&](int tile, int& m_tile, int& n_tile, int& seg, int& kb0, int& nkb) {
+    seg = 0; kb0 = 0; nkb = num_kb;
+    int lt = tile;
+    if (k_seg) {
+      seg = tile / seg_tiles;
+      lt = tile - seg * seg_tiles;
+      kb0 = k_seg[seg] / BLOCK_K;
+      nkb = (k_seg[seg + 1] - k_seg[seg]) / BLOCK_K;
+    }
+    m_tile = lt / n_tiles;
+    n_tile = lt - m_tile * n_tiles;
+  };
   const uint32_t stage_tx = A_STAGE_BYTES + (uint32_t)block_n * BLOCK_K * 2;
 
   if (threadIdx.x == 0) {
@@ -337,16 +353,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       int issued = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m_tile = tile / n_tiles, n_tile = tile % n_tiles;
+        int m_tile, n_tile, seg, kb0, nkb;
+        decode(tile, m_tile, n_tile, seg, kb0, nkb);
         const int e = tile_expert ? tile_expert[m_tile] : 0;
         const int b_row = MODE == EPI_SWIGLU ? e * 2 * N + n_tile * 128 : e * N + n_tile * block_n;
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kq = 0; kq < nkb; ++kq) {
+          const int kb = kb0 + kq;
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
           mbar_expect_tx(full_bar(stage), stage_tx);
           const uint32_t sa = base + stage * SB;
           // fault injection (tests only): the copies of K block `withhold_kb` of this CTA's first tile are never issued,
           // so the stage never fills and the waits downstream run out
-          if (!(withhold_kb >= 0 && tile == (int)blockIdx.x && kb == withhold_kb)) {
+          if (!(withhold_kb >= 0 && tile == (int)blockIdx.x && kq == withhold_kb)) {
             tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BLOCK_K, m_tile * BLOCK_M);
             tma_load_2d(sa + A_STAGE_BYTES, &tmap_b, full_bar(stage), kb * BLOCK_K, b_row);
             if (MODE == EPI_SWIGLU)     // second half of the B tile: the up rows of the same 128 hidden units (box = 128 rows)
@@ -380,7 +398,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)acc * MAX_BLOCK_N;
-        for (int kb = 0; kb < num_kb; ++kb) {
+        int m_tile_, n_tile_, seg_, kb0_, nkb;
+        decode(tile, m_tile_, n_tile_, seg_, kb0_, nkb);
+        for (int kb = 0; kb < nkb; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, wait_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + stage * SB;
@@ -420,7 +440,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const int m_tile = tile / n_tiles, n_tile = tile % n_tiles;
+      int m_tile, n_tile, seg, kb0_, nkb;
+      decode(tile, m_tile, n_tile, seg, kb0_, nkb);
       // warp-uniform outcome: the tensor-memory loads below need the whole warp
       if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, abort_flag, wait_limit))) { ok = false; break; }
       tc_fence_after();
@@ -490,6 +511,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           __syncwarp();
         }
       }
+      // weight-gradient mode: problem `seg` owns its own rows of C; an empty K range leaves zeros
+      Epilogue epl = ep;
+      if (MODE == EPI_F32 && k_seg) epl.C = reinterpret_cast<float*>(ep.C) + (size_t)seg * M_max * ep.ldc;
+      const bool zero_acc = MODE == EPI_F32 && k_seg && nkb == 0;
       int ch = (MODE == EPI_SWIGLU || EWQ == 4) ? n_chunks : half;
       if (ch < n_chunks) tmem_ld32_issue(taddr + ch * 32, ra);
       // two register buffers: while one chunk is processed the next chunk's tensor-memory load is in flight
@@ -497,14 +522,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);     // in flight together with the tensor-memory load
         tmem_ld_wait(ra);
         if (ch + EWQ < n_chunks) tmem_ld32_issue(taddr + (ch + EWQ) * 32, rb);
-        if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
+        if (zero_acc) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ra[i] = 0u;
+        }
+        if (f32_out(MODE)) epi_softplus32<MODE>(epl, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, ra, bq, lane);
         else if (row_ok) epi_store32<MODE>(ep, out_row, tok_row, n_base + ch * 32, N, ra, scale, bq);
         ch += EWQ;
         if (ch >= n_chunks) break;
         load_bias<MODE>(ep, n_base + ch * 32, N, bq);
         tmem_ld_wait(rb);
         if (ch + EWQ < n_chunks) tmem_ld32_issue(taddr + (ch + EWQ) * 32, ra);
-        if (f32_out(MODE)) epi_softplus32<MODE>(ep, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
+        if (zero_acc) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) rb[i] = 0u;
+        }
+        if (f32_out(MODE)) epi_softplus32<MODE>(epl, out_stage + (warp - 2) * 1024, m_tile * BLOCK_M + quarter * 32, M_valid, n_base + ch * 32, N, rb, bq, lane);
         else if (row_ok) epi_store32<MODE>(ep, out_row, tok_row, n_base + ch * 32, N, rb, scale, bq);
         ch += EWQ;
       }
@@ -587,7 +620,33 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
   const long long max_tiles = (long long)((M_max + BLOCK_M - 1) / BLOCK_M) * n_tiles;
   const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
   kern<<<grid, threads_of(epi.mode), smem_bytes, st>>>(ta, tb, M_max, N, Kd, block_n, idesc, tile_expert, num_m_tiles_dev, epi, status,
-                                                            test_stall ? WAIT_LIMIT_TEST : WAIT_LIMIT, test_stall ? 1 : -1);
+                                                            test_stall ? WAIT_LIMIT_TEST : WAIT_LIMIT, test_stall ? 1 : -1, nullptr, 0);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// Grouped weight gradient on the tensor cores: C[s][P, Q] (fp32) = sum over the rows r in [seg[s], seg[s+1]) of Xt[p, r] Yt[q, r].
+// Xt [P, ld], Yt [Q, ld]: the activations transposed, so the contracted token rows are contiguous; seg: n_seg + 1 device offsets,
+// multiples of 64 (the padded expert segments); rows outside every segment are never read.
+cudaError_t launch_gemm_tc_wgrad(const void* Xt, const void* Yt, int ld, const int32_t* seg, int n_seg, int P, int Q, float* C,
+                                 int32_t* status, cudaStream_t st) {
+  const int block_n = Q >= MAX_BLOCK_N ? MAX_BLOCK_N : (Q + 31) / 32 * 32;
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, Xt, (uint64_t)P, (uint64_t)ld, (uint64_t)ld, BLOCK_M)) return cudaErrorInvalidValue;
+  if (!make_tmap(&tb, Yt, (uint64_t)Q, (uint64_t)ld, (uint64_t)ld, (uint32_t)block_n)) return cudaErrorInvalidValue;
+  const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(block_n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+  int num_sms = 0;
+  cudaError_t e = current_device_sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
+  const int smem_bytes = smem_bytes_of(EPI_F32);
+  e = cudaFuncSetAttribute(gemm_tc_kernel<EPI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e != cudaSuccess) return e;
+  const int n_tiles = (Q + block_n - 1) / block_n;
+  const long long max_tiles = (long long)n_seg * ((P + BLOCK_M - 1) / BLOCK_M) * n_tiles;
+  const int grid = (int)(max_tiles < num_sms ? max_tiles : num_sms);
+  const Epilogue epi{EPI_F32, C, Q, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
+  gemm_tc_kernel<EPI_F32><<<grid, threads_of(EPI_F32), smem_bytes, st>>>(ta, tb, P, Q, ld, block_n, idesc, nullptr, nullptr, epi, status,
+                                                                        WAIT_LIMIT, -1, seg, n_seg);
   count_launch();
   return cudaGetLastError();
 }

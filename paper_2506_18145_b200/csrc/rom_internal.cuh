@@ -151,6 +151,13 @@ cudaError_t launch_gemm_tc(const void* A, int lda, const void* Bw, int ldb, int 
                            int M_max, int N, int Kd, const int32_t* tile_expert, const int32_t* num_m_tiles_dev,
                            const Epilogue& epi, int32_t* status, cudaStream_t st, bool test_stall = false);
 
+// Grouped weight gradient on the tensor cores (bf16): C[s][P, Q] fp32 = sum over rows r of segment s of Xt[p, r] Yt[q, r];
+// Xt [P, ld], Yt [Q, ld] bf16 (activations transposed); seg: n_seg + 1 device row offsets, multiples of 64.
+cudaError_t launch_gemm_tc_wgrad(const void* Xt, const void* Yt, int ld, const int32_t* seg, int n_seg, int P, int Q, float* C,
+                                 int32_t* status, cudaStream_t st);
+// out[c][r] = scale[r] * in[r][c] for in [R, C] (scale may be nullptr); out has row pitch ldo >= R.
+cudaError_t launch_transpose_scaled(int dtype, const void* in, void* out, int R, int C, int ldo, const float* scale, cudaStream_t st);
+
 // row_of_assign == nullptr (top-1, rows already in token order): row t of XZp belongs to token t.
 // Zs (K > 1 only): [T, d_inner], SiLU of the Gate Proj rows summed over the K slots.
 cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,
