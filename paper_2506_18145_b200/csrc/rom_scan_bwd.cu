@@ -12,8 +12,12 @@
 // the states (dDelta, du, the forward y for the gate's derivative) are shuffles over those lanes; sums over channels
 // (dB, dC) are shuffles over the 8 channels of a warp, shared-memory atomics over the block and one global atomic per
 // (step, state) and block; dA and dD accumulate in registers over the sequence and leave with one atomic per thread.
-// All arithmetic is fp32 with the accurate exp / expm1 (both storage types): this is the first, plain version of
-// the kernel; its time is not tuned.
+// A long sequence with few channels is cut into coarse chunks that run in parallel, as in the forward scan: both
+// recurrences are linear, the states' forward in time and the state gradients' backward in time.  A pre-pass runs, per
+// coarse chunk, the state recurrence from a zero state (end state, sum of Delta) and the gradient recurrence from a
+// zero gradient (the gradient leaving the chunk's start); a chain kernel composes them into the true state at the start
+// and the true gradient at the end of every coarse chunk; the two kernels above then run once per coarse chunk.
+// All arithmetic is fp32 with the accurate exp / expm1 (both storage types).
 #include "rom_internal.cuh"
 
 namespace rom {
@@ -32,6 +36,11 @@ struct BwdArgs {
   float* ckpt;        // [B, nck, De, 16]
   int L, De, nck;
   int ldz;            // row pitch (elements) of z and dz
+  // coarse chunks (blockIdx.z): chunk j covers steps [j Lc, (j+1) Lc); Lc is a multiple of CK.  ncc == 1: the whole sequence.
+  int Lc, ncc;
+  const float* h_in;  // [B, ncc, De, 16] state at the start of every coarse chunk (ncc > 1)
+  const float* g_in;  // [B, ncc, De, 16] state gradient at the end of every coarse chunk (ncc > 1)
+  float* h_end; float* q_start; float* sum_delta;     // pre-pass outputs: [B, ncc, De, 16] x 2 and [B, ncc, De]
 };
 
 __device__ __forceinline__ float sigmoid_f(float v) { return 1.0f / (1.0f + expf(-v)); }
@@ -45,13 +54,16 @@ scan_ckpt_kernel(const BwdArgs p) {
   const size_t b = blockIdx.y;
   if (c >= p.De) return;
   const T* __restrict__ u = static_cast<const T*>(p.u);
+  const int cj = blockIdx.z;
+  const int t_lo = cj * p.Lc, t_hi = min(t_lo + p.Lc, p.L);
   float a[4], h[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     a[i] = p.A[(size_t)c * NST + 4 * q + i];
-    h[i] = p.h0 ? p.h0[(b * p.De + c) * NST + 4 * q + i] : 0.0f;
+    if (p.ncc > 1) h[i] = p.h_in[((b * p.ncc + cj) * p.De + c) * NST + 4 * q + i];
+    else h[i] = p.h0 ? p.h0[(b * p.De + c) * NST + 4 * q + i] : 0.0f;
   }
-  for (int t = 0; t < p.L; ++t) {
+  for (int t = t_lo; t < t_hi; ++t) {
     if ((t % CK) == 0)
       *reinterpret_cast<float4*>(p.ckpt + ((b * p.nck + t / CK) * p.De + c) * NST + 4 * q) = make_float4(h[0], h[1], h[2], h[3]);
     const size_t e = (b * p.L + t) * p.De + c;
@@ -97,16 +109,19 @@ scan_bwd_kernel(const BwdArgs p) {
   T* __restrict__ du = static_cast<T*>(p.du);
   T* __restrict__ dz = static_cast<T*>(p.dz);
 
+  const int cj = blockIdx.z;
+  const int k_lo = cj * (p.Lc / CK), k_hi = min(k_lo + p.Lc / CK, p.nck);
   float a[4], g[4], dAacc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     a[i] = p.A[(size_t)cc * NST + 4 * q + i];
-    g[i] = p.dh_last ? p.dh_last[(b * p.De + cc) * NST + 4 * q + i] : 0.0f;
+    if (p.ncc > 1) g[i] = p.g_in[((b * p.ncc + cj) * p.De + cc) * NST + 4 * q + i];
+    else g[i] = p.dh_last ? p.dh_last[(b * p.De + cc) * NST + 4 * q + i] : 0.0f;
   }
   const float Dc = p.D ? p.D[cc] : 0.0f;
   float dDacc = 0.0f;
 
-  for (int k = p.nck - 1; k >= 0; --k) {
+  for (int k = k_hi - 1; k >= k_lo; --k) {
     const int t0 = k * CK;
     const int nt = min(CK, p.L - t0);
     // ---- stage the chunk's inputs; e = dout * SiLU(z) is the gradient arriving at y
@@ -233,17 +248,113 @@ scan_bwd_kernel(const BwdArgs p) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       atomicAdd(p.dA + (size_t)c * NST + 4 * q + i, dAacc[i]);
-      if (p.dh0) p.dh0[(b * p.De + c) * NST + 4 * q + i] = g[i];
+      if (p.dh0 && cj == 0) p.dh0[(b * p.De + c) * NST + 4 * q + i] = g[i];
     }
     if (q == 0 && p.dD) atomicAdd(p.dD + c, dDacc);
   }
+}
+
+
+// Pre-pass of the chunk-parallel form, one coarse chunk per blockIdx.z: from a zero state the chunk's end state and sum
+// of Delta; from a zero gradient the gradient that leaves the chunk's start (g <- a_t (g + C_t e_t), t descending).
+template <typename T, bool ZOH>
+__global__ void __launch_bounds__(BT)
+scan_bwd_prepass_kernel(const BwdArgs p) {
+  const int tid = threadIdx.x, cl = tid >> 2, q = tid & 3;
+  const int c = blockIdx.x * BCH + cl;
+  const size_t b = blockIdx.y;
+  if (c >= p.De) return;
+  const int cj = blockIdx.z;
+  const int t_lo = cj * p.Lc, t_hi = min(t_lo + p.Lc, p.L);
+  const T* __restrict__ u = static_cast<const T*>(p.u);
+  const T* __restrict__ dy = static_cast<const T*>(p.dy);
+  const T* __restrict__ z = static_cast<const T*>(p.z);
+  float a[4], h[4] = {0.0f, 0.0f, 0.0f, 0.0f}, g[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) a[i] = p.A[(size_t)c * NST + 4 * q + i];
+  float sd = 0.0f;
+  for (int t = t_lo; t < t_hi; ++t) {
+    const size_t e = (b * p.L + t) * p.De + c;
+    const float dl = p.delta[e], uu = to_f32(u[e]);
+    const float4 B4 = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
+    const float bv[4] = {B4.x, B4.y, B4.z, B4.w};
+    sd += dl;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float x = dl * a[i];
+      const float bb = ZOH ? expm1f(x) / a[i] * bv[i] : dl * bv[i];
+      h[i] = fmaf(expf(x), h[i], bb * uu);
+    }
+  }
+  for (int t = t_hi - 1; t >= t_lo; --t) {
+    const size_t e = (b * p.L + t) * p.De + c;
+    const float dl = p.delta[e];
+    float ev = to_f32(dy[e]);
+    if (z) { const float zz = to_f32(z[(b * p.L + t) * p.ldz + c]); ev *= zz * sigmoid_f(zz); }
+    const float4 C4 = *reinterpret_cast<const float4*>(p.Cm + (b * p.L + t) * NST + 4 * q);
+    const float cv[4] = {C4.x, C4.y, C4.z, C4.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) g[i] = fmaf(cv[i], ev, g[i]) * expf(dl * a[i]);
+  }
+  const size_t o = ((b * p.ncc + cj) * p.De + c) * NST + 4 * q;
+  *reinterpret_cast<float4*>(p.h_end + o) = make_float4(h[0], h[1], h[2], h[3]);
+  *reinterpret_cast<float4*>(p.q_start + o) = make_float4(g[0], g[1], g[2], g[3]);
+  if (q == 0) p.sum_delta[(b * p.ncc + cj) * p.De + c] = sd;
+}
+
+// Composes the coarse chunks (both recurrences are linear): with P_j = exp(A sum_delta_j),
+//   h_in[0] = h0,  h_in[j+1] = P_j h_in[j] + h_end[j];   g_in[ncc-1] = dh_last,  g_in[j-1] = P_j g_in[j] + q_start[j].
+__global__ void __launch_bounds__(256)
+scan_bwd_chain_kernel(const float* __restrict__ A, const float* __restrict__ h0, const float* __restrict__ dh_last,
+                      const float* __restrict__ h_end, const float* __restrict__ q_start, const float* __restrict__ sum_delta,
+                      float* __restrict__ h_in, float* __restrict__ g_in, int B, int De, int ncc) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)B * De * NST) return;
+  const int n = (int)(i % NST);
+  const int c = (int)((i / NST) % De);
+  const size_t b = (size_t)(i / ((long long)NST * De));
+  const float a = A[(size_t)c * NST + n];
+  float h = h0 ? h0[i] : 0.0f;
+  for (int j = 0; j < ncc; ++j) {
+    const size_t sq = b * ncc + j;
+    h_in[(sq * De + c) * NST + n] = h;
+    h = fmaf(expf(a * sum_delta[sq * De + c]), h, h_end[(sq * De + c) * NST + n]);
+  }
+  float g = dh_last ? dh_last[i] : 0.0f;
+  for (int j = ncc - 1; j >= 0; --j) {
+    const size_t sq = b * ncc + j;
+    g_in[(sq * De + c) * NST + n] = g;
+    g = fmaf(expf(a * sum_delta[sq * De + c]), g, q_start[(sq * De + c) * NST + n]);
+  }
+}
+
+// Coarse chunks per sequence: 1 when batch x channels already give about 2048 blocks' worth of work, else enough chunks
+// (each a multiple of CK steps, at least 4 CK) to get there.  A function of the sizes only (workspace sizing = launch).
+int coarse_chunks(int B, int De, int L, int* Lc_out) {
+  const long long blocks1 = (long long)B * ((De + BCH - 1) / BCH);
+  int ncc = 1;
+  if (blocks1 < 1024) {
+    ncc = (int)((2048 + blocks1 - 1) / blocks1);
+    const int max_ncc = (L + 4 * CK - 1) / (4 * CK);
+    if (ncc > max_ncc) ncc = max_ncc;
+    if (ncc < 1) ncc = 1;
+  }
+  int Lc = (L + ncc - 1) / ncc;
+  Lc = (Lc + CK - 1) / CK * CK;
+  ncc = (L + Lc - 1) / Lc;
+  *Lc_out = Lc;
+  return ncc;
 }
 
 }  // namespace
 
 size_t scan_bwd_ws_bytes(int B, int De, int L) {
   const size_t nck = (size_t)(L + CK - 1) / CK;
-  return align_up(sizeof(float) * (size_t)B * nck * De * NST, 256);
+  int Lc = 0;
+  const int ncc = coarse_chunks(B, De, L, &Lc);
+  size_t floats = (size_t)B * nck * De * NST;
+  if (ncc > 1) floats += (size_t)B * ncc * De * (4 * NST + 1);
+  return align_up(sizeof(float) * floats, 256);
 }
 
 cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void* u, const float* delta, const float* A,
@@ -251,14 +362,36 @@ cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void
                                  const float* dh_last, void* du, float* ddelta, float* dA, float* dBm, float* dCm, float* dD,
                                  void* dz, float* dh0, float* ckpt, int ldz, cudaStream_t st) {
   const int nck = (c.L + CK - 1) / CK;
-  const BwdArgs a{dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0, ckpt, c.L, c.d_inner, nck, ldz};
+  int Lc = 0;
+  const int ncc = coarse_chunks(c.B, c.d_inner, c.L, &Lc);
+  const size_t n_fine = (size_t)c.B * nck * c.d_inner * NST, n_coarse = (size_t)c.B * ncc * c.d_inner * NST;
+  float* h_end = ckpt + n_fine;
+  float* q_start = h_end + n_coarse;
+  float* h_in = q_start + n_coarse;
+  float* g_in = h_in + n_coarse;
+  float* sum_delta = g_in + n_coarse;
+  const BwdArgs a{dy, u, delta, A, Bm, Cm, D, z, h0, dh_last, du, ddelta, dA, dBm, dCm, dD, dz, dh0, ckpt, c.L, c.d_inner, nck, ldz,
+                  Lc, ncc, h_in, g_in, h_end, q_start, sum_delta};
   cudaError_t e = cudaMemsetAsync(dA, 0, sizeof(float) * (size_t)c.d_inner * NST, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(dBm, 0, sizeof(float) * (size_t)c.B * c.L * NST, st);
   if (e == cudaSuccess) e = cudaMemsetAsync(dCm, 0, sizeof(float) * (size_t)c.B * c.L * NST, st);
   if (e == cudaSuccess && dD) e = cudaMemsetAsync(dD, 0, sizeof(float) * (size_t)c.d_inner, st);
   if (e != cudaSuccess) return e;
-  const dim3 grid((c.d_inner + BCH - 1) / BCH, c.B);
+  const dim3 grid((c.d_inner + BCH - 1) / BCH, c.B, ncc);
   const bool zoh = c.disc_mode == 0, bf = c.dtype == ROM_BF16;
+  if (ncc > 1) {
+    if (bf) {
+      if (zoh) scan_bwd_prepass_kernel<__nv_bfloat16, true><<<grid, BT, 0, st>>>(a); else scan_bwd_prepass_kernel<__nv_bfloat16, false><<<grid, BT, 0, st>>>(a);
+    } else {
+      if (zoh) scan_bwd_prepass_kernel<float, true><<<grid, BT, 0, st>>>(a); else scan_bwd_prepass_kernel<float, false><<<grid, BT, 0, st>>>(a);
+    }
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const long long n_thr = (long long)c.B * c.d_inner * NST;
+    scan_bwd_chain_kernel<<<(unsigned)((n_thr + 255) / 256), 256, 0, st>>>(A, h0, dh_last, h_end, q_start, sum_delta, h_in, g_in, c.B, c.d_inner, ncc);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
   if (bf) {
     if (zoh) scan_ckpt_kernel<__nv_bfloat16, true><<<grid, BT, 0, st>>>(a); else scan_ckpt_kernel<__nv_bfloat16, false><<<grid, BT, 0, st>>>(a);
   } else {
