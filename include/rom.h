@@ -181,7 +181,7 @@ ROM_API int rom_scan(const rom_config *cfg, const void *u, const float *delta, c
  *   dBm, dCm [B, L, d_state], dD [d_inner] (NULL exactly when D is) fp32, each the sum over everything that shares the
  *   parameter (dA and dD over sequences and steps; dBm, dCm over channels) -- accumulated with floating-point atomics,
  *   so their last bits vary from run to run;  dh0 [B, d_inner, d_state] fp32 or NULL.
- * ws: rom_scan_backward_workspace_size(cfg) bytes (the state at the start of every 32 steps).  All arithmetic fp32.
+ * ws: rom_scan_backward_workspace_size(cfg) bytes (the state at the start of every 16 steps, plus the chunk states of the chunk-parallel form).  All arithmetic fp32.
  * Uses cfg->B, L, d_inner, d_state, dtype, disc_mode.                                                              */
 ROM_API int rom_scan_backward_workspace_size(const rom_config *cfg, size_t *bytes);
 ROM_API int rom_scan_backward(const rom_config *cfg, const void *dy, const void *u, const float *delta, const float *A,

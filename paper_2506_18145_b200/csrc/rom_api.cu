@@ -548,11 +548,22 @@ int rom_layer_backward(const rom_config* cfg, const rom_weights* w, const void* 
   ROM_CUDA(launch_softplus_bwd(c.dtype, ddelta, D32, W + bl.dpre, g->db_dt, T, De, st));
   ROM_CUDA(launch_transpose(c.dtype, w->W_dt, W + bl.WdtT, 1, De, R, st));
   ROM_CUDA(gemm(W + bl.dpre, De, W + bl.WdtT, De, 1, 0, T, R, De, nullptr, nullptr, store_to(W + bl.dxdbl, R + 2 * N)));      // d(delta) into columns [0, R)
-  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dpre, De, W + lay.delta_r, R, nullptr, nullptr, 1, T, De, R, g->dW_dt, st));
+  // weight gradient of a shared projection (a sum over all tokens): tensor path = the plain GEMM over transposed
+  // activations (row pitch padded to 64 tokens; the tail of the last K block is filled with zeros by the tensor map)
+  const int Tp = (int)align_up((size_t)T, 64);
+  auto shared_wgrad = [&](const void* X, int P, const void* Y, int Q, float* C) -> cudaError_t {
+    if (!tc) return launch_wgrad(c.dtype, X, P, Y, Q, nullptr, nullptr, 1, T, P, Q, C, st);
+    cudaError_t e = launch_transpose_scaled(c.dtype, X, W + bl.Xt, T, P, Tp, nullptr, st);
+    if (e == cudaSuccess) e = launch_transpose_scaled(c.dtype, Y, W + bl.Yt, T, Q, Tp, nullptr, st);
+    if (e == cudaSuccess) e = launch_gemm_tc(W + bl.Xt, Tp, W + bl.Yt, Tp, 1, P, Q, T, nullptr, nullptr,
+                                             Epilogue{EPI_F32, C, Q, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr}, status, st);
+    return e;
+  };
+  ROM_CUDA(shared_wgrad(W + bl.dpre, De, W + lay.delta_r, R, g->dW_dt));
   ROM_CUDA(launch_pack_bc(c.dtype, dBm, dCm, W + bl.dxdbl, T, R, N, st));
   ROM_CUDA(launch_transpose(c.dtype, w->W_x, W + bl.WxT, 1, R + 2 * N, De, st));
   ROM_CUDA(gemm(W + bl.dxdbl, R + 2 * N, W + bl.WxT, R + 2 * N, 1, 0, T, De, R + 2 * N, nullptr, nullptr, store_to(W + bl.dU2, De)));
-  ROM_CUDA(launch_wgrad(c.dtype, W + bl.dxdbl, R + 2 * N, W + lay.U, De, nullptr, nullptr, 1, T, R + 2 * N, De, g->dW_x, st));
+  ROM_CUDA(shared_wgrad(W + bl.dxdbl, R + 2 * N, W + lay.U, De, g->dW_x));
 
   // ---- conv, reversed (dU = scan part + x Proj part)
   ROM_CUDA(cudaMemsetAsync(g->dw_conv, 0, sizeof(float) * (size_t)c.d_conv * De, st));

@@ -6,7 +6,7 @@
 //           g += C_t e_t;  dC_t = sum_c e_t h_t;  dA-bar = g h_{t-1};  db = g u_t;  du_t = sum_n g b + D e_t;  g <- a_t g.
 //
 // The reverse sweep needs h_{t-1} and h_t at every step.  A first kernel runs the recurrence forward and keeps the
-// state at the start of every chunk of 32 steps (checkpoints in the workspace).  The second kernel walks the chunks
+// state at the start of every chunk of 16 steps (checkpoints in the workspace).  The second kernel walks the chunks
 // backwards: it recomputes the chunk's states from its checkpoint into shared memory, then sweeps the chunk in
 // reverse.  A thread owns 4 of the 16 states of one channel of one sequence (4 adjacent lanes per channel): sums over
 // the states (dDelta, du, the forward y for the gate's derivative) are shuffles over those lanes; sums over channels
@@ -24,7 +24,7 @@ namespace rom {
 namespace {
 
 constexpr int NST = 16;
-constexpr int CK = 32;            // steps per chunk
+constexpr int CK = 16;            // steps per chunk (16: four blocks fit an SM's shared memory)
 constexpr int BCH = 32;           // channels per block
 constexpr int BT = BCH * 4;       // threads per block
 constexpr size_t BWD_SMEM = sizeof(float4) * CK * BT + sizeof(float) * CK * (8 * BCH + 4 * NST);
