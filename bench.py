@@ -214,6 +214,19 @@ def run_stage(args, s):
         nbytes = 0
         # forward recompute (in_proj) + data and weight gradients of the two grouped projections
         extra = {"flops": 2.0 * s.T * s.K * s.d_model * s.d_inner * (2 + 2 * 3), "d_ff": None}
+    elif args.stage == "mamba2":
+        # RoM on a Mamba2-style block at the workload's widths, headdim 64 (first version: the scalar-per-head recurrence runs
+        # on the selective-scan kernel as a special case)
+        headdim = 64
+        p = synth.make_mamba2_inputs(s, headdim)
+        d = {k: (None if v is None else v.to(dev)) for k, v in p.items()}
+        w2 = rb.make_mamba2_weights(d)
+        ws = torch.empty(rb.mamba2_workspace_size(cfg, headdim), dtype=torch.uint8, device=dev)
+        out = torch.empty_like(d["x"])
+        call = lambda: rb.rom_mamba2_layer_forward(cfg, headdim, w2, d["x"], out, None, None, None, ws)
+        nbytes = 0
+        Wd = 2 * s.d_inner + 2 * s.d_state + s.d_inner // headdim
+        extra = {"flops": 2.0 * s.T * s.K * s.d_model * (Wd + s.d_inner), "d_ff": None}
     elif args.stage == "step":
         # single-token step at the workload's widths, 64 sequences generating in lock-step; states stay on the device
         sb = s.replace(B=64, L=1)
@@ -307,7 +320,7 @@ def main():
     ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
                     help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
                          "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
-    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn", "step", "backward"],
+    ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn", "step", "backward", "mamba2"],
                     help="layer: the whole forward (the benchmark); scan / route / ffn / step: that entry point alone, timed in isolation "
                          "at the workload's shape (kernel studies and ncu captures; prints a short JSON line)")
     args = ap.parse_args()

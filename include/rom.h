@@ -282,6 +282,36 @@ ROM_API int rom_ffn_moe_forward(const rom_config *cfg, int32_t d_ff, const void 
                         const void *x, const int32_t *topk_idx, const float *gates, void *out,
                         void *ws, size_t ws_bytes, void *stream);
 
+/* Routing Mamba on a Mamba2-style block (Section 5.2, "RoM on other linear recurrent architectures"; Section 5.4, first
+ * insight: for blocks with a unified design all major projection layers become experts under the shared routing;
+ * Appendix A.2: the deployment "follows the same logic" as on Mamba).  The paper prints no equations for this variant:
+ * the block is the published Mamba2 block with one B/C group, and per token t
+ *   [z | x | B | C | dt]_t = sum_i 1_i X_t W_in,i           (indicator only; widths D_e | D_e | N | N | heads)
+ *   (x, B, C) <- SiLU(causal depthwise conv(x, B, C) + b_conv);   dt_h = softplus(dt_h + dt_bias_h)
+ *   per head h (headdim channels):  H_t = exp(dt_h A_h) H_{t-1} + dt_h x_t (x) B_t,   y_t = C_t H_t + D_h x_t
+ *   y^_t = (y_t * SiLU(z_t)) / sqrt(mean_c (y_t * SiLU(z_t))_c^2 + 1e-5) * w_norm
+ *   O_t = sum_i R_i(X_t) y^_t W_out,i
+ * with the router, top-K, gates and permutation of rom_route.  Shared by all experts: conv, A, D, dt_bias, w_norm.
+ *   headdim : channels per head; d_inner / headdim heads, a multiple of 8.  cfg->dt_rank, disc_mode and
+ *             small_proj_experts are not used; d_state must be 16, d_conv 2..4.
+ *   x, out  : [B, L, d_model] dtype;  ws: rom_mamba2_workspace_size(cfg, headdim) bytes.                            */
+typedef struct {                  /* read-only device pointers */
+  const void  *W_r;               /* [E, d_model]                               dtype */
+  const float *b_r;               /* [E] or NULL */
+  const void  *W_in;              /* [E, 2*d_inner + 2*d_state + heads, d_model] dtype  rows z | x | B | C | dt */
+  const void  *w_conv;            /* [d_conv, d_inner + 2*d_state]              dtype  tap d_conv-1 = current token */
+  const float *b_conv;            /* [d_inner + 2*d_state] or NULL */
+  const float *dt_bias;           /* [heads] or NULL */
+  const float *A;                 /* [heads], strictly negative */
+  const float *D;                 /* [heads] or NULL */
+  const float *w_norm;            /* [d_inner] */
+  const void  *W_out;             /* [E, d_model, d_inner]                      dtype */
+} rom_mamba2_weights;
+ROM_API int rom_mamba2_workspace_size(const rom_config *cfg, int32_t headdim, size_t *bytes);
+ROM_API int rom_mamba2_layer_forward(const rom_config *cfg, int32_t headdim, const rom_mamba2_weights *w, const void *x,
+                             void *out, int32_t *topk_idx_out, float *gates_out, int32_t *counts_out,
+                             void *ws, size_t ws_bytes, void *stream);
+
 /* Profiling aid: the same launch sequence as rom_layer_forward with a CUDA event recorded on
  * `stream` between stages; synchronises the stream and writes the device time of each stage in
  * milliseconds to stage_ms (host out, at least rom_num_stages() floats).  Stage i is named

@@ -26,7 +26,7 @@ EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "
            "rom_num_stages", "rom_stage_name", "rom_route_noalloc", "rom_route_balance",
            "rom_ffn_moe_workspace_size", "rom_ffn_moe_forward", "rom_layer_step", "rom_layer_forward_host",
            "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward",
-           "rom_layer_backward_workspace_size", "rom_layer_backward")
+           "rom_layer_backward_workspace_size", "rom_layer_backward", "rom_mamba2_workspace_size", "rom_mamba2_layer_forward")
 
 
 class RomConfig(ctypes.Structure):
@@ -43,6 +43,11 @@ class RomWeights(ctypes.Structure):
 class RomGrads(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("dW_r", "db_r", "dW_inz", "dw_conv", "db_conv", "dW_x", "dW_dt", "db_dt", "dA", "dD", "dW_out")]
+
+
+class RomMamba2Weights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("W_r", "b_r", "W_in", "w_conv", "b_conv", "dt_bias", "A", "D", "w_norm", "W_out")]
 
 
 class RomError(RuntimeError):
@@ -69,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.rom_debug_check.argtypes = [cfgp, vp, ctypes.c_size_t, vp]
         L.rom_scan_backward_workspace_size.argtypes = [cfgp, szp]
         L.rom_layer_backward_workspace_size.argtypes = [cfgp, szp]
+        L.rom_mamba2_workspace_size.argtypes = [cfgp, ctypes.c_int32, szp]
+        L.rom_mamba2_layer_forward.argtypes = [cfgp, ctypes.c_int32, ctypes.POINTER(RomMamba2Weights), vp, vp, i32p, vp, i32p, vp, ctypes.c_size_t, vp]
         L.rom_layer_backward.argtypes = [cfgp, ctypes.POINTER(RomWeights), vp, vp, vp, ctypes.POINTER(RomGrads), vp, ctypes.c_size_t, vp]
         L.rom_scan_backward.argtypes = [cfgp] + [vp] * 19 + [ctypes.c_size_t, vp]
         L.rom_route.argtypes = [cfgp, vp, vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp, ctypes.c_size_t, vp]
@@ -140,7 +147,7 @@ def scan_workspace_size(cfg: RomConfig) -> int:
     rc = lib().rom_scan_workspace_size(ctypes.byref(cfg), ctypes.byref(n))
     if rc != ROM_OK:
         raise RomError(rc, "rom_scan_workspace_size", "rom_debug_check", "rom_scan_backward_workspace_size", "rom_scan_backward",
-           "rom_layer_backward_workspace_size", "rom_layer_backward")
+           "rom_layer_backward_workspace_size", "rom_layer_backward", "rom_mamba2_workspace_size", "rom_mamba2_layer_forward")
     return int(n.value)
 
 
@@ -225,6 +232,26 @@ def rom_layer_backward(cfg, weights: RomWeights, x, dout, dx, grads: RomGrads, w
                                   ws.numel() if ws is not None else 0, _stream(stream))
     if check and rc != ROM_OK:
         raise RomError(rc, "rom_layer_backward")
+    return rc
+
+
+def mamba2_workspace_size(cfg: RomConfig, headdim: int) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().rom_mamba2_workspace_size(ctypes.byref(cfg), int(headdim), ctypes.byref(n))
+    if rc != ROM_OK:
+        raise RomError(rc, "rom_mamba2_workspace_size")
+    return int(n.value)
+
+
+def make_mamba2_weights(w: Dict[str, Optional[torch.Tensor]]) -> RomMamba2Weights:
+    return RomMamba2Weights(*[_ptr(w.get(n)) for n, _ in RomMamba2Weights._fields_])
+
+
+def rom_mamba2_layer_forward(cfg, headdim, weights: RomMamba2Weights, x, out, topk_idx_out, gates_out, counts_out, ws, stream=None, check=True) -> int:
+    rc = lib().rom_mamba2_layer_forward(ctypes.byref(cfg), int(headdim), ctypes.byref(weights), _ptr(x), _ptr(out), _ptr(topk_idx_out),
+                                        _ptr(gates_out), _ptr(counts_out), _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream))
+    if check and rc != ROM_OK:
+        raise RomError(rc, "rom_mamba2_layer_forward")
     return rc
 
 

@@ -160,3 +160,35 @@ def make_scan_inputs(B: int, L: int, d_inner: int, d_state: int, dtype: str, see
     out["z"] = _randn(sb + _TID["z"], (B, L, d_inner)).to(dt) if with_z else None
     out["h0"] = _randn(sb + _TID["h0"], (B, d_inner, d_state)) if with_h0 else None
     return out
+
+
+def make_mamba2_inputs(shape: RomShape, headdim: int) -> Dict[str, Optional[torch.Tensor]]:
+    """x and every weight of one RoM layer on a Mamba2-style block, O(1) outputs at every stage ("unit" scaling):
+    projection std 1/sqrt(fan_in), conv taps std 0.5, router std 2/sqrt(D_m), A_h = -(0.5 + rand) * (1 + h mod 8),
+    D ~ N(0,1), dt bias = softplus^-1(dt0) with dt0 log-uniform in [1e-3, 1e-1], norm weight 1 + 0.1 N(0,1).
+    Layouts: W_in[E, 2 D_e + 2 N + heads, D_m] rows z | x | B | C | dt; w_conv[k, D_e + 2 N]; W_out[E, D_m, D_e]."""
+    s = shape
+    dt = torch_dtype(s)
+    De, N, Dm = s.d_inner, s.d_state, s.d_model
+    H = De // headdim
+    W = 2 * De + 2 * N + H
+    sb = s.seed_base + 300
+    out: Dict[str, Optional[torch.Tensor]] = {}
+    out["x"] = _randn(sb + 1, (s.B, s.L, Dm)).to(dt)
+    out["W_r"] = _randn(sb + 2, (s.E, Dm), 2.0 / math.sqrt(Dm)).to(dt)
+    out["W_in"] = _randn(sb + 3, (s.E, W, Dm), 1.0 / math.sqrt(Dm)).to(dt)
+    out["w_conv"] = _randn(sb + 4, (s.d_conv, De + 2 * N), 0.5).to(dt)
+    out["b_conv"] = _randn(sb + 5, (De + 2 * N,), 0.1)
+    u01 = _rand(sb + 6, (H,)).double()
+    dt0 = torch.exp(u01 * (math.log(1e-1) - math.log(1e-3)) + math.log(1e-3))
+    out["dt_bias"] = (dt0 + torch.log(-torch.expm1(-dt0))).float()
+    out["A"] = (-(0.5 + _rand(sb + 7, (H,))) * (1.0 + (torch.arange(H) % 8).float())).contiguous()
+    out["D"] = _randn(sb + 8, (H,))
+    out["w_norm"] = 1.0 + 0.1 * _randn(sb + 9, (De,))
+    out["W_out"] = _randn(sb + 10, (s.E, Dm, De), 1.0 / math.sqrt(De)).to(dt)
+    if s.router_bias_scale is None:
+        out["b_r"] = None
+    else:
+        e = torch.arange(s.E, dtype=torch.float64)
+        out["b_r"] = (-s.router_bias_scale * 1.2 * torch.log(e + 1.0)).float()
+    return out
