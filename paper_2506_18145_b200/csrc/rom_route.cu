@@ -356,20 +356,21 @@ route_scatter(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ 
 __global__ void __launch_bounds__(256)
 route_scatter_gather(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ chunk_base,
                      const int32_t* __restrict__ offsets, const int32_t* __restrict__ pad_offsets,
-                     int T_tokens, int E, int K,
+                     int T_tokens, int E, int K, int n_chunks,
                      int32_t* __restrict__ perm, int32_t* __restrict__ inv_perm,
                      int32_t* __restrict__ row_of_assign, int32_t* __restrict__ assign_of_row,
                      const uint4* __restrict__ x, uint4* __restrict__ x_perm, int vec_per_row) {
   __shared__ int32_t rows_s[kChunkTokens * kMaxK];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int chunk = blockIdx.x;
-  if (warp == 0) {
+  // blocks beyond the last chunk (the grid never drops below one block per SM) only help with the padding rows
+  if (chunk < n_chunks && warp == 0) {
     int my_row[kMaxK];
     scatter_chunk(topk_idx, chunk_base, offsets, pad_offsets, T_tokens, E, K, chunk, lane, perm, inv_perm, row_of_assign, assign_of_row, my_row);
     for (int k = 0; k < K; ++k) rows_s[lane * K + k] = my_row[k];
   }
   __syncthreads();
-  const int n_tok = min(kChunkTokens, T_tokens - chunk * kChunkTokens);
+  const int n_tok = chunk < n_chunks ? min(kChunkTokens, T_tokens - chunk * kChunkTokens) : 0;
   for (int j = warp; j < n_tok; j += 8) {
     const uint4* src = x + (size_t)(chunk * kChunkTokens + j) * vec_per_row;
     for (int v0 = 0; v0 < vec_per_row; v0 += 32 * 8) {
@@ -544,7 +545,11 @@ static cudaError_t launch_scatter(const rom_config& c, const int32_t* idx_ws, in
   int32_t* roa = reinterpret_cast<int32_t*>(ws + lay.row_of_assign);
   int32_t* aor = reinterpret_cast<int32_t*>(ws + lay.assign_of_row);
   if (x != nullptr) {
-    route_scatter_gather<<<(int)lay.n_chunks, 256, 0, st>>>(idx_ws, chunk_base, offs, poffs, (int)lay.T, c.E, c.K, perm, inv_perm, roa, aor,
+    int num_sms = 0;
+    const cudaError_t e = current_device_sm_count(&num_sms);
+    if (e != cudaSuccess) return e;
+    const int grid = (int)lay.n_chunks > num_sms ? (int)lay.n_chunks : num_sms;
+    route_scatter_gather<<<grid, 256, 0, st>>>(idx_ws, chunk_base, offs, poffs, (int)lay.T, c.E, c.K, (int)lay.n_chunks, perm, inv_perm, roa, aor,
                                                            reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(ws + lay.x_perm),
                                                            (int)((size_t)c.d_model * lay.esz / 16));
   } else {
