@@ -317,6 +317,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--simt", action="store_true", help="run the projections on the fp32-FMA bisecting path")
+    ap.add_argument("--fused-small", action="store_true", help="conv, x Proj and dt Proj as the one fused kernel instead of three launches")
     ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
                     help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
                          "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
@@ -352,7 +353,8 @@ def main():
     routed_small = args.small_proj == "routed"
     p = synth.make_inputs(s, routed_small=routed_small)
     d = {k: (None if v is None else v.to(dev)) for k, v in p.items()}
-    cfg = rb.config_from_shape(s, flags=rb.ROM_FLAG_SIMT_GEMM if args.simt else 0, small_proj_experts=s.E if routed_small else 0)
+    cfg = rb.config_from_shape(s, flags=(rb.ROM_FLAG_SIMT_GEMM if args.simt else 0) | (rb.ROM_FLAG_FUSED_SMALL if args.fused_small else 0),
+                               small_proj_experts=s.E if routed_small else 0)
     weights = rb.make_weights(d)
     ws = rb.alloc_workspace(cfg, dev)
     x_dev = d["x"]

@@ -76,6 +76,11 @@ typedef struct {
                                  before the first kernel and compared after the last.  A violation is latched as
                                  ROM_ERR_DEBUG_CHECK.  The workspace is larger with this flag (rom_workspace_size and
                                  rom_workspace_find take it into account); two more small launches per call.      */
+#define ROM_FLAG_FUSED_SMALL 8 /* tensor path at top-1 with the shared x Proj / dt Proj: run the short conv, the x Proj and the
+                                 dt Proj + softplus as ONE tcgen05 kernel (U written once and never re-read, delta kept on
+                                 the SM) instead of three launches.  Same results up to rounding.  Off by default: as
+                                 measured it is slower than the three launches (instruction-issue bound on one CTA per
+                                 128 tokens); ignored where the sizes do not fit (d_r > 128, d_r + 2 D_s > 160)          */
 #define ROM_FLAG_TEST_STALL 4 /* fault injection for tests of the device-side timeout path (tensor path only): the
                                  first grouped projection withholds the copies of one operand stage per CTA and
                                  every device wait gives up after 2^14 polls instead of 2^22, so the call returns

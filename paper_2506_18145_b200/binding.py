@@ -19,6 +19,7 @@ ROM_F32, ROM_BF16 = 0, 1
 ROM_FLAG_SIMT_GEMM = 1
 ROM_FLAG_DEBUG_CHECKS = 2
 ROM_FLAG_TEST_STALL = 4
+ROM_FLAG_FUSED_SMALL = 8
 ROM_OK = 0
 
 EXPORTS = ("rom_workspace_size", "rom_route", "rom_scan", "rom_layer_forward", "rom_workspace_find",

@@ -80,7 +80,7 @@ int check_config(const rom_config* c, int which) {
   if (!c) return ROM_ERR_INVALID_ARG;
   if (c->dtype != ROM_F32 && c->dtype != ROM_BF16) return ROM_ERR_INVALID_ARG;
   if (c->B < 1 || c->L < 1) return ROM_ERR_INVALID_ARG;
-  if ((c->flags & ~(ROM_FLAG_SIMT_GEMM | ROM_FLAG_DEBUG_CHECKS | ROM_FLAG_TEST_STALL)) != 0) return ROM_ERR_INVALID_ARG;
+  if ((c->flags & ~(ROM_FLAG_SIMT_GEMM | ROM_FLAG_DEBUG_CHECKS | ROM_FLAG_TEST_STALL | ROM_FLAG_FUSED_SMALL)) != 0) return ROM_ERR_INVALID_ARG;
   if (which != 2) {
     if (c->E < 1 || c->K < 1 || c->K > c->E) return ROM_ERR_INVALID_ARG;
     if (c->E > kMaxE || c->K > kMaxK) return ROM_ERR_UNSUPPORTED;
@@ -326,6 +326,16 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
                 in_token_order ? reinterpret_cast<const int32_t*>(W + lay.assign_of_row) : nullptr, nullptr};
   ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_inz, Dm, c.E, (int64_t)2 * De * Dm, (int)lay.rows_max, 2 * De, Dm, tile_expert, num_m_tiles, e_in));
   ROM_STAGE_DONE();
+  // S4 + S5 + S6 as one kernel (opt-in): tensor path, top-1 (rows already in token order), shared x Proj / dt Proj
+  const bool fused_small = in_token_order && !conv_state && c.small_proj_experts <= 1 && (c.flags & ROM_FLAG_FUSED_SMALL) &&
+                           fused_conv_xdt_supported(c);
+  if (fused_small) {
+    ROM_CUDA(launch_fused_conv_xdt(c, W + lay.XZp, 2 * De, w->w_conv, w->b_conv, w->W_x, w->W_dt, w->b_dt, W + lay.U, W + lay.delta_r,
+                                   reinterpret_cast<float*>(W + lay.Bm), reinterpret_cast<float*>(W + lay.Cm), W + lay.Delta, status, st));
+    ROM_STAGE_DONE();      // "conv": the fused kernel's time is reported here
+    ROM_STAGE_DONE();      // "x_proj"
+    ROM_STAGE_DONE();      // "dt_proj"
+  } else {
   // S4: un-permute + sum over selected experts + conv + SiLU
   if (conv_state)
     ROM_CUDA(launch_conv_step(c, W + lay.XZp, in_token_order ? nullptr : row_of_assign, w->w_conv, w->b_conv, conv_state, W + lay.U,
@@ -368,6 +378,7 @@ int layer_forward_impl(const rom_config* cfg, const rom_weights* w, const void* 
       ROM_STAGE_DONE();
     }
   }
+  }      // !fused_small
   // S7 + S8 + S9: scan, gate, re-permute
   // K = 1: the gate row of a token is its Gate Proj row in expert order; K > 1: the summed rows from S4
   const char* zbase = c.K == 1 ? W + lay.XZp + (size_t)De * lay.esz : W + lay.Zs;

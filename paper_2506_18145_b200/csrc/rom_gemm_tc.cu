@@ -20,18 +20,13 @@
 // TMEM and returns.
 //
 // Every TMA load here is a plain single-CTA load (no thread-block clusters).
-#include <cuda.h>
-
-#include "rom_internal.cuh"
+#include "rom_tc_ptx.cuh"
 
 namespace rom {
 namespace {
 
 constexpr int NUM_EPI_WARPS_C = 8;
-constexpr int BLOCK_M = 128;
-constexpr int BLOCK_K = 64;            // 64 bf16 = 128 bytes = one swizzle row
 constexpr int MAX_BLOCK_N = 256;
-constexpr int UMMA_K = 16;
 constexpr int MAX_STAGES = 4;
 constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;          // 16 KB
 constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;      // 32 KB
@@ -58,88 +53,6 @@ __host__ __device__ constexpr int stages_of(int mode) { return f32_out(mode) ? 3
 __host__ __device__ constexpr int out_stage_bytes_of(int mode) { return f32_out(mode) ? epi_warps_of(mode) * 32 * 32 * 4 : 0; }
 __host__ __device__ constexpr int smem_bytes_of(int mode) {
   return stages_of(mode) * stage_bytes_of(mode) + 1024 /*alignment slack*/ + 256 /*barriers*/ + out_stage_bytes_of(mode);
-}
-constexpr uint32_t WAIT_LIMIT = 1u << 22;        // try_wait polls before a wait gives up (a few seconds)
-constexpr uint32_t WAIT_LIMIT_TEST = 1u << 14;   // the same under the fault-injection flag (milliseconds)
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the limit is reached or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
-  for (uint32_t i = 0; i < limit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-}
-// Waits for the outstanding tensor-memory load; the loaded registers pass through the statement so that
-// nothing that reads them can be scheduled ahead of the wait.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :: "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements),
-// written by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset),
-// the leading byte offset is unused for swizzled K-major layouts, descriptor version 1, layout type 2.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3ffffu) >> 4);          // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                            // leading byte offset (ignored)
-  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
-  d |= (uint64_t)1 << 46;                            // version
-  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
-  return d;
 }
 
 // Bias of the 32 columns [n0, n0+32) (EPI_SOFTPLUS only), requested before the accumulator chunk is waited for.
@@ -243,41 +156,6 @@ __device__ __forceinline__ void epi_softplus32(const Epilogue& ep, float* sw, in
     }
   }
   __syncwarp();
-}
-
-// Softplus output op for sixteen epilogue warps: a warp owns two adjacent 32-column chunks of its 32 rows.  Every lane
-// activates and rounds its row of a chunk to bf16 and stages it (swizzled 16-byte pieces, 128 bytes per row for the two
-// chunks); after the second chunk the warp writes whole 128-byte row segments, four rows per store instruction.
-// stage: 32 rows x 8 pieces of 16 bytes.  piece0: first piece of this chunk (0 or 4).
-__device__ __forceinline__ void softplus_stage_bf16(uint4* stage, int piece0, const uint32_t (&r)[32], const float4 (&bq)[8], int lane) {
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float4 b0 = bq[2 * j], b1 = bq[2 * j + 1];
-    uint4 q;
-    __nv_bfloat162 h0 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j]) + b0.x), softplus_bf16(__uint_as_float(r[8 * j + 1]) + b0.y));
-    __nv_bfloat162 h1 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j + 2]) + b0.z), softplus_bf16(__uint_as_float(r[8 * j + 3]) + b0.w));
-    __nv_bfloat162 h2 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j + 4]) + b1.x), softplus_bf16(__uint_as_float(r[8 * j + 5]) + b1.y));
-    __nv_bfloat162 h3 = __floats2bfloat162_rn(softplus_bf16(__uint_as_float(r[8 * j + 6]) + b1.z), softplus_bf16(__uint_as_float(r[8 * j + 7]) + b1.w));
-    q.x = *reinterpret_cast<uint32_t*>(&h0); q.y = *reinterpret_cast<uint32_t*>(&h1);
-    q.z = *reinterpret_cast<uint32_t*>(&h2); q.w = *reinterpret_cast<uint32_t*>(&h3);
-    stage[lane * 8 + ((piece0 + j) ^ (lane & 7))] = q;
-  }
-}
-// n0: column of piece 0; pieces at or beyond n_pieces (0, 4 or 8 valid) or beyond N are not written.
-template <int MODE>
-__device__ __forceinline__ void softplus_flush_bf16(const Epilogue& ep, const uint4* stage, int row0, int M_valid, int n0, int N,
-                                                    int n_pieces, int lane) {
-  const int p = lane & 7;
-  const int n = n0 + 8 * p;
-#pragma unroll
-  for (int r4 = 0; r4 < 8; ++r4) {
-    const int R = r4 * 4 + (lane >> 3);
-    const uint4 q = stage[R * 8 + (p ^ (R & 7))];
-    if (row0 + R < M_valid && p < n_pieces && n < N) {
-      const int orow = MODE == EPI_SOFTPLUS_ROWS ? __ldg(ep.row_token + row0 + R) : row0 + R;
-      if (orow >= 0) *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(ep.C) + (size_t)orow * ep.ldc + n) = q;
-    }
-  }
 }
 
 template <int MODE>
@@ -558,35 +436,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
-}
-
-// ---------------------------------------------------------------------------------------------- host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;      // resolving the driver symbol is idempotent; a benign race
-  if (fn) return fn;
-  void* p = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess)
-    return nullptr;
-  fn = reinterpret_cast<EncodeTiledFn>(p);
-  return fn;
-}
-
-// 2-D bf16 row-major [rows, cols] (cols contiguous, row stride ld elements); box = 64 cols x box_rows.
-bool make_tmap(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {ld * 2};
-  cuuint32_t box[2] = {BLOCK_K, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace

@@ -158,6 +158,13 @@ cudaError_t launch_gemm_tc_wgrad(const void* Xt, const void* Yt, int ld, const i
 // out[c][r] = scale[r] * in[r][c] for in [R, C] (scale may be nullptr); out has row pitch ldo >= R.
 cudaError_t launch_transpose_scaled(int dtype, const void* in, void* out, int R, int C, int ldo, const float* scale, cudaStream_t st);
 
+// Conv + SiLU, x Proj and dt Proj + softplus as one tcgen05 kernel (bf16, rows of HZ in token order, shared small layers):
+// U, delta_r, Bm, Cm, Delta as the three separate launches leave them.  fused_conv_xdt_supported says whether the sizes fit.
+bool fused_conv_xdt_supported(const rom_config& c);
+cudaError_t launch_fused_conv_xdt(const rom_config& c, const void* HZ, int ldh, const void* w_conv, const float* b_conv, const void* W_x,
+                                  const void* W_dt, const float* b_dt, void* U, void* delta_r, float* Bm, float* Cm, void* Delta,
+                                  int32_t* status, cudaStream_t st);
+
 // row_of_assign == nullptr (top-1, rows already in token order): row t of XZp belongs to token t.
 // Zs (K > 1 only): [T, d_inner], SiLU of the Gate Proj rows summed over the K slots.
 cudaError_t launch_conv(const rom_config& c, const void* XZp, const int32_t* row_of_assign, const void* w_conv,

@@ -59,7 +59,7 @@ def _cfg(**kw):
     (dict(K=5), -1), (dict(K=0), -1), (dict(E=0), -1), (dict(E=65, K=1), -2), (dict(E=16, K=9), -2),
     (dict(d_model=100), -1), (dict(d_inner=200), -1), (dict(d_state=8), -2), (dict(d_conv=5), -2),
     (dict(d_conv=0), -1), (dict(dt_rank=0), -1), (dict(dt_rank=24), -2), (dict(B=0), -1), (dict(L=0), -1),
-    (dict(gate_mode=2), -1), (dict(disc_mode=3), -1), (dict(flags=8), -1),
+    (dict(gate_mode=2), -1), (dict(disc_mode=3), -1), (dict(flags=16), -1),
 ])
 def test_layer_forward_rejects_bad_configs_on_the_host(L, kw, code):
     cfg = _cfg(**kw)

@@ -486,3 +486,33 @@ def test_device_wait_that_runs_out_is_reported_and_the_workspace_stays_usable():
     ref, im = oracle_layer(s, p)
     np.testing.assert_array_equal(good.idx.cpu().numpy(), im["idx"])
     assert_close(np64(out), ref, TOL["bf16"], "out after a timed-out call")
+
+
+# ---------------------------------------------------------------------------------------------- fused conv + x Proj + dt Proj
+@pytest.mark.parametrize("kw", [
+    dict(E=8, K=1, B=3, L=130),                                   # ragged last row tile, several sequences inside one tile
+    dict(E=4, K=1, B=1, L=700, d_conv=3, dt_rank=32),
+    dict(E=4, K=1, B=2, L=257, d_conv=2, dt_rank=64, d_inner=512),
+    dict(E=2, K=1, B=5, L=33, dt_rank=128, d_inner=320),           # d_r = 128: two K blocks of the dt Proj; D_e not a multiple of 256
+])
+def test_fused_small_projections_match_the_three_launches_and_the_oracle(kw):
+    """ROM_FLAG_FUSED_SMALL runs conv + x Proj + dt Proj as one tcgen05 kernel (top-1, tensor path); the default is three
+    launches.  Both against the oracle (taps U, B, C, Delta and the output), and against each other."""
+    s = small_shape(**kw)
+    check_layer(s, "unit")
+    check_layer(s, "unit", flags=rb.ROM_FLAG_FUSED_SMALL)
+    p = synth.make_inputs(s, recipe="unit")
+    a = GpuLayer(s, p, flags=rb.ROM_FLAG_FUSED_SMALL)
+    out_a = a.forward().clone()
+    n_fused = rb.last_launch_count()
+    b = GpuLayer(s, p)
+    out_b = b.forward()
+    assert rb.last_launch_count() == n_fused + 2
+    tdt = synth.torch_dtype(s)
+    assert_close(np64(a.tap("U", tdt, s.d_inner)), np64(b.tap("U", tdt, s.d_inner)), 1e-2, "U fused vs unfused")
+    assert_close(np64(a.tap("Delta", tdt, s.d_inner)), np64(b.tap("Delta", tdt, s.d_inner)), 1e-2, "Delta fused vs unfused")
+    assert_close(np64(out_a), np64(out_b), 1e-2, "out fused vs unfused")
+
+
+def test_fused_small_projections_small_bf16_config():
+    check_layer(synth.CONFIGS["small_bf16"], "unit", with_D=False, flags=rb.ROM_FLAG_FUSED_SMALL)
