@@ -17,7 +17,8 @@
 // coarse chunk, the state recurrence from a zero state (end state, sum of Delta) and the gradient recurrence from a
 // zero gradient (the gradient leaving the chunk's start); a chain kernel composes them into the true state at the start
 // and the true gradient at the end of every coarse chunk; the two kernels above then run once per coarse chunk.
-// All arithmetic is fp32 with the accurate exp / expm1 (both storage types).
+// All arithmetic is fp32; the fp32 configuration uses the accurate exp / expm1, the bf16 one a single ex2.approx per state
+// and step (exp(x) - 1 by subtraction: with Delta A down to -5e-4 that is still good to a few 1e-4 relative).
 #include "rom_internal.cuh"
 
 namespace rom {
@@ -45,6 +46,15 @@ struct BwdArgs {
 
 __device__ __forceinline__ float sigmoid_f(float v) { return 1.0f / (1.0f + expf(-v)); }
 
+// exp(x) and exp(x) - 1
+template <bool PRECISE>
+__device__ __forceinline__ void exp_and_expm1(float x, float& ex, float& em1) {
+  if (PRECISE) { ex = expf(x); em1 = expm1f(x); }
+  else { ex = ex2_ftz(1.4426950408889634f * x); em1 = ex - 1.0f; }
+}
+template <bool PRECISE>
+__device__ __forceinline__ float exp_only(float x) { return PRECISE ? expf(x) : ex2_ftz(1.4426950408889634f * x); }
+
 // Forward pass that only records the state at the start of every chunk.
 template <typename T, bool ZOH>
 __global__ void __launch_bounds__(BT)
@@ -63,18 +73,33 @@ scan_ckpt_kernel(const BwdArgs p) {
     if (p.ncc > 1) h[i] = p.h_in[((b * p.ncc + cj) * p.De + c) * NST + 4 * q + i];
     else h[i] = p.h0 ? p.h0[(b * p.De + c) * NST + 4 * q + i] : 0.0f;
   }
-  for (int t = t_lo; t < t_hi; ++t) {
-    if ((t % CK) == 0)
-      *reinterpret_cast<float4*>(p.ckpt + ((b * p.nck + t / CK) * p.De + c) * NST + 4 * q) = make_float4(h[0], h[1], h[2], h[3]);
-    const size_t e = (b * p.L + t) * p.De + c;
-    const float dl = p.delta[e], uu = to_f32(u[e]);
-    const float4 B4 = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
-    const float bv[4] = {B4.x, B4.y, B4.z, B4.w};
+  constexpr bool PRECISE = sizeof(T) == 4;
+  float ia[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float x = dl * a[i];
-      const float bb = ZOH ? expm1f(x) / a[i] * bv[i] : dl * bv[i];
-      h[i] = fmaf(expf(x), h[i], bb * uu);
+  for (int i = 0; i < 4; ++i) ia[i] = 1.0f / a[i];
+  for (int t4 = t_lo; t4 < t_hi; t4 += 4) {       // CK is a multiple of 4: a checkpoint falls on the first step of a group
+    float dl[4], uu[4];
+    float4 B4[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {                 // the group's loads first
+      const int t = min(t4 + j, t_hi - 1);
+      const size_t e = (b * p.L + t) * p.De + c;
+      dl[j] = p.delta[e]; uu[j] = to_f32(u[e]);
+      B4[j] = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
+    }
+    if ((t4 % CK) == 0)
+      *reinterpret_cast<float4*>(p.ckpt + ((b * p.nck + t4 / CK) * p.De + c) * NST + 4 * q) = make_float4(h[0], h[1], h[2], h[3]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (t4 + j >= t_hi) break;
+      const float bv[4] = {B4[j].x, B4[j].y, B4[j].z, B4[j].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float ex, em1;
+        exp_and_expm1<PRECISE>(dl[j] * a[i], ex, em1);
+        const float bb = ZOH ? em1 * ia[i] * bv[i] : dl[j] * bv[i];
+        h[i] = fmaf(ex, h[i], bb * uu[j]);
+      }
     }
   }
 }
@@ -120,6 +145,10 @@ scan_bwd_kernel(const BwdArgs p) {
   }
   const float Dc = p.D ? p.D[cc] : 0.0f;
   float dDacc = 0.0f;
+  constexpr bool PRECISE = sizeof(T) == 4;
+  float ia[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) ia[i] = 1.0f / a[i];
 
   for (int k = k_hi - 1; k >= k_lo; --k) {
     const int t0 = k * CK;
@@ -154,9 +183,10 @@ scan_bwd_kernel(const BwdArgs p) {
       float ys = 0.0f;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const float x = dl * a[i];
-        const float bb = ZOH ? expm1f(x) / a[i] * s_B[r][4 * q + i] : dl * s_B[r][4 * q + i];
-        h[i] = fmaf(expf(x), h[i], bb * uu);
+        float ex, em1;
+        exp_and_expm1<PRECISE>(dl * a[i], ex, em1);
+        const float bb = ZOH ? em1 * ia[i] * s_B[r][4 * q + i] : dl * s_B[r][4 * q + i];
+        h[i] = fmaf(ex, h[i], bb * uu);
         ys = fmaf(s_C[r][4 * q + i], h[i], ys);
       }
       hbuf[r][tid] = make_float4(h[0], h[1], h[2], h[3]);
@@ -181,14 +211,15 @@ scan_bwd_kernel(const BwdArgs p) {
         const float Bv = s_B[r][4 * q + i], Cv = s_C[r][4 * q + i];
         g[i] = fmaf(Cv, ev, g[i]);
         dCp[i] = ev * hc[i];
-        const float x = dl * a[i], ex = expf(x);
+        float ex, em1;
+        exp_and_expm1<PRECISE>(dl * a[i], ex, em1);
         float dx = g[i] * hp[i] * ex;              // through A-bar = exp(x)
         if (ZOH) {
-          const float em1 = expm1f(x), ia = 1.0f / a[i];
-          dx = fmaf(g[i] * uu * Bv * ia, ex, dx);  // through expm1(x)
-          dAacc[i] = fmaf(g[i] * uu * Bv, -em1 * ia * ia, dAacc[i]);
-          dBp[i] = g[i] * uu * em1 * ia;
-          duv = fmaf(g[i] * em1 * ia, Bv, duv);
+          const float gub = g[i] * uu * Bv * ia[i], ge = g[i] * em1 * ia[i];
+          dx = fmaf(gub, ex, dx);                  // through expm1(x)
+          dAacc[i] = fmaf(gub, -em1 * ia[i], dAacc[i]);
+          dBp[i] = ge * uu;
+          duv = fmaf(ge, Bv, duv);
           dd = fmaf(dx, a[i], dd);
         } else {
           dBp[i] = g[i] * uu * dl;
@@ -207,16 +238,30 @@ scan_bwd_kernel(const BwdArgs p) {
         s_du[r][cl] = fmaf(Dc, ev, duv);
         dDacc = fmaf(ev, uu, dDacc);
       }
-      // sums over channels: the 8 channels of the warp by shuffles, then the block's warps by shared-memory atomics
+      // sums over channels: the 8 channels of a warp hold 8 values each (4 dB, 4 dC of the lane's states); three exchange
+      // steps halve the values a lane keeps while adding its partner's, so every lane ends with ONE fully reduced value
+      // (7 shuffles instead of 24), then the block's warps meet in shared-memory atomics
+      {
+        float v[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float vb = c_ok ? dBp[i] : 0.0f, vc = dCp[i];
+        for (int i = 0; i < 4; ++i) { v[i] = c_ok ? dBp[i] : 0.0f; v[4 + i] = dCp[i]; }
+        const bool b2 = lane & 4, b3 = lane & 8, b4 = lane & 16;
+        float w4[4], w2[2];
 #pragma unroll
-        for (int o = 4; o < 32; o <<= 1) {
-          vb += __shfl_xor_sync(0xffffffffu, vb, o);
-          vc += __shfl_xor_sync(0xffffffffu, vc, o);
+        for (int i = 0; i < 4; ++i) {
+          const float send = b2 ? v[i] : v[4 + i], keep = b2 ? v[4 + i] : v[i];
+          w4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
         }
-        if (lane < 4) { atomicAdd(&s_dB[r][4 * q + i], vb); atomicAdd(&s_dC[r][4 * q + i], vc); }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const float send = b3 ? w4[i] : w4[2 + i], keep = b3 ? w4[2 + i] : w4[i];
+          w2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+        const float send = b4 ? w2[0] : w2[1], keep = b4 ? w2[1] : w2[0];
+        const float tot = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        const int idx = (b2 ? 4 : 0) + (b3 ? 2 : 0) + (b4 ? 1 : 0);      // which of the 8 values this lane ended with
+        float* dst = idx < 4 ? &s_dB[r][4 * q + idx] : &s_dC[r][4 * q + (idx - 4)];
+        atomicAdd(dst, tot);
       }
     }
     __syncthreads();
@@ -272,29 +317,54 @@ scan_bwd_prepass_kernel(const BwdArgs p) {
   float a[4], h[4] = {0.0f, 0.0f, 0.0f, 0.0f}, g[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
   for (int i = 0; i < 4; ++i) a[i] = p.A[(size_t)c * NST + 4 * q + i];
-  float sd = 0.0f;
-  for (int t = t_lo; t < t_hi; ++t) {
-    const size_t e = (b * p.L + t) * p.De + c;
-    const float dl = p.delta[e], uu = to_f32(u[e]);
-    const float4 B4 = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
-    const float bv[4] = {B4.x, B4.y, B4.z, B4.w};
-    sd += dl;
+  constexpr bool PRECISE = sizeof(T) == 4;
+  float ia[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float x = dl * a[i];
-      const float bb = ZOH ? expm1f(x) / a[i] * bv[i] : dl * bv[i];
-      h[i] = fmaf(expf(x), h[i], bb * uu);
+  for (int i = 0; i < 4; ++i) ia[i] = 1.0f / a[i];
+  float sd = 0.0f;
+  for (int t4 = t_lo; t4 < t_hi; t4 += 4) {
+    float dl[4], uu[4];
+    float4 B4[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int t = min(t4 + j, t_hi - 1);
+      const size_t e = (b * p.L + t) * p.De + c;
+      dl[j] = p.delta[e]; uu[j] = to_f32(u[e]);
+      B4[j] = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (t4 + j >= t_hi) break;
+      const float bv[4] = {B4[j].x, B4[j].y, B4[j].z, B4[j].w};
+      sd += dl[j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float ex, em1;
+        exp_and_expm1<PRECISE>(dl[j] * a[i], ex, em1);
+        const float bb = ZOH ? em1 * ia[i] * bv[i] : dl[j] * bv[i];
+        h[i] = fmaf(ex, h[i], bb * uu[j]);
+      }
     }
   }
-  for (int t = t_hi - 1; t >= t_lo; --t) {
-    const size_t e = (b * p.L + t) * p.De + c;
-    const float dl = p.delta[e];
-    float ev = to_f32(dy[e]);
-    if (z) { const float zz = to_f32(z[(b * p.L + t) * p.ldz + c]); ev *= zz * sigmoid_f(zz); }
-    const float4 C4 = *reinterpret_cast<const float4*>(p.Cm + (b * p.L + t) * NST + 4 * q);
-    const float cv[4] = {C4.x, C4.y, C4.z, C4.w};
+  for (int t4 = t_hi - 1; t4 >= t_lo; t4 -= 4) {
+    float dl[4], ev[4];
+    float4 C4[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) g[i] = fmaf(cv[i], ev, g[i]) * expf(dl * a[i]);
+    for (int j = 0; j < 4; ++j) {
+      const int t = max(t4 - j, t_lo);
+      const size_t e = (b * p.L + t) * p.De + c;
+      dl[j] = p.delta[e];
+      ev[j] = to_f32(dy[e]);
+      if (z) { const float zz = to_f32(z[(b * p.L + t) * p.ldz + c]); ev[j] *= zz * sigmoid_f(zz); }
+      C4[j] = *reinterpret_cast<const float4*>(p.Cm + (b * p.L + t) * NST + 4 * q);
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (t4 - j < t_lo) break;
+      const float cv[4] = {C4[j].x, C4[j].y, C4[j].z, C4[j].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) g[i] = fmaf(cv[i], ev[j], g[i]) * exp_only<PRECISE>(dl[j] * a[i]);
+    }
   }
   const size_t o = ((b * p.ncc + cj) * p.De + c) * NST + 4 * q;
   *reinterpret_cast<float4*>(p.h_end + o) = make_float4(h[0], h[1], h[2], h[3]);
