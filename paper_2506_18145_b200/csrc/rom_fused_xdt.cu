@@ -3,11 +3,11 @@
 //   U = SiLU(conv(H) + b_conv),  (delta | B | C) = U W_x^T,  Delta = softplus(delta W_dt^T + b_dt).
 // U is written to HBM once and never read back by these steps, delta never leaves the SM.
 //
-// One CTA owns a tile of 128 tokens and all D_e channels.  576 threads: a TMA producer warp, an MMA-issuing warp
+// One CTA owns a tile of up to 128 tokens (the token count is spread evenly over the SMs) and all D_e channels.  576 threads: a TMA producer warp, an MMA-issuing warp
 // (tcgen05, accumulators in tensor memory) and 16 worker warps that change role with the phase:
 //   phase 1  per block of 64 channels the producer brings the 131 x 64 block of H (the tile's rows and the three
 //            before them) and the matching 64 columns of W_x by TMA, three blocks ahead; the workers compute conv +
-//            SiLU from shared memory (16 channels of one token per thread), write it to U and, as bf16 in the
+//            SiLU from shared memory (8 channels of two consecutive tokens per thread), write it to U and, as bf16 in the
 //            128-byte-swizzled K-major layout the tensor core expects, into an operand stage; the MMA thread
 //            accumulates the 128 x (d_r + 2 D_s) x Proj tile over all channel blocks.
 //   phase 2  workers read that tile from tensor memory: B, C go to HBM in fp32, delta is rounded to bf16 and laid
@@ -56,6 +56,7 @@ struct FusedArgs {
   int T, L, De, R, N, k;
   int block_n1;                 // x Proj tile width: R + 2N rounded up to 32
   int block_n3;                 // dt Proj tile width: min(256, De rounded up to 32)
+  int rows_cta;                 // tokens per CTA (<= 128, a multiple of 8): chosen so that every SM gets the same share
 };
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -73,6 +74,7 @@ __device__ __forceinline__ uint4 pack8(const float (&v)[8]) {
   return q;
 }
 
+template <int KCONV>
 __global__ void __launch_bounds__(F_THREADS, 1)
 fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_wx,
                       const __grid_constant__ CUtensorMap tmap_wdt, const FusedArgs p, uint32_t idesc1, uint32_t idesc3, int32_t* __restrict__ status, uint32_t wait_limit) {
@@ -88,18 +90,19 @@ fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_c
   auto fullA = [&](int s) { return bars + 8u * s; };
   auto fullB = [&](int s) { return bars + 8u * (F_STAGES + s); };
   auto empty1 = [&](int s) { return bars + 8u * (2 * F_STAGES + s); };
-  const uint32_t d1_full = bars + 8u * (3 * F_STAGES);
-  const uint32_t a2_ready = bars + 8u * (3 * F_STAGES + 1);
-  auto full3 = [&](int s) { return bars + 8u * (3 * F_STAGES + 2 + s); };
-  auto empty3 = [&](int s) { return bars + 8u * (4 * F_STAGES + 2 + s); };
-  auto tfull = [&](int a) { return bars + 8u * (5 * F_STAGES + 2 + a); };
-  auto tempty = [&](int a) { return bars + 8u * (5 * F_STAGES + 4 + a); };
-  const uint32_t drain_bar = bars + 8u * (5 * F_STAGES + 6);
+  constexpr int BB = 3 * F_STAGES;
+  const uint32_t d1_full = bars + 8u * BB;
+  const uint32_t a2_ready = bars + 8u * (BB + 1);
+  auto full3 = [&](int s) { return bars + 8u * (BB + 2 + s); };
+  auto empty3 = [&](int s) { return bars + 8u * (BB + 2 + F_STAGES + s); };
+  auto tfull = [&](int a) { return bars + 8u * (BB + 2 + 2 * F_STAGES + a); };
+  auto tempty = [&](int a) { return bars + 8u * (BB + 4 + 2 * F_STAGES + a); };
+  const uint32_t drain_bar = bars + 8u * (BB + 6 + 2 * F_STAGES);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem + F_STAGE_REGION + F_A2_BYTES + 8 * F_NUM_BARS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * BLOCK_M;
+  const int m0 = blockIdx.x * p.rows_cta;
   const int nkc = p.De / BLOCK_K;                              // channel blocks of the x Proj contraction
   const int kb3 = (p.R + BLOCK_K - 1) / BLOCK_K;               // K blocks of the dt Proj
   const int nt3 = (p.De + p.block_n3 - 1) / p.block_n3;        // channel tiles of the dt Proj
@@ -130,9 +133,9 @@ fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_c
   const uint32_t tmem_base = *tmem_holder;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer: W_x blocks, then W_dt blocks
+    // ------------------------------------------------------------------ TMA producer: H and W_x blocks, then W_dt blocks
     if (lane == 0) {
-      uint32_t last_bar[F_STAGES] = {0, 0, 0}, last_par[F_STAGES] = {0, 0, 0};
+      uint32_t last_bar[F_STAGES] = {}, last_par[F_STAGES] = {};
       int n_last = 0;
       int stage = 0; uint32_t phase = 0;
       bool ok = true;
@@ -145,7 +148,7 @@ fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_c
         last_bar[n_last % F_STAGES] = fullB(stage); last_par[n_last % F_STAGES] = phase; ++n_last;
         if (++stage == F_STAGES) { stage = 0; phase ^= 1u; }
       }
-      // the dt Proj stages reuse the x Proj stages: wait until the last x Proj MMA has read them
+      // the dt Proj stages reuse the phase 1 region: wait until the last x Proj MMA has read it (the workers are done with H by then)
       if (ok && !mbar_wait(d1_full, 0, abort_flag, wait_limit)) ok = false;
       stage = 0; phase = 0;
       for (int nt = 0; nt < nt3 && ok; ++nt) {
@@ -224,68 +227,67 @@ fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_c
     const int wt = w * 32 + lane;                 // 0..511
     bool ok = true;
 
-    // ---- phase 1: conv + SiLU of the tile, one 64-channel block after the other
+    // ---- phase 1: conv + SiLU of the tile, one 64-channel block after the other.  A thread owns 8 channels of two
+    // consecutive tokens: the five rows of H it needs are unpacked once and serve both tokens.
     {
-      const int r = wt >> 2, cg = wt & 3;         // token row of the tile; 16 channels [16 cg, 16 cg + 16) of the block
-      const int tok = m0 + r;
-      const bool valid = tok < p.T;
-      const int t = valid ? tok % p.L : 0;        // position inside its sequence (the conv does not cross sequences)
-      __nv_bfloat16* urow = p.U + (size_t)(valid ? tok : 0) * p.De + 16 * cg;
-      const uint32_t sw0 = (uint32_t)r * 128u + (uint32_t)(((2 * cg) ^ (r & 7)) << 4);       // swizzled 16-byte slots of the row
-      const uint32_t sw1 = (uint32_t)r * 128u + (uint32_t)(((2 * cg + 1) ^ (r & 7)) << 4);
+      const int cg = wt & 7, r0 = (wt >> 3) * 2;  // 16-byte channel group of the block; first of the thread's two rows
+      bool valid[2];
+      int tpos[2];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int tok = m0 + r0 + i;
+        valid[i] = r0 + i < p.rows_cta && tok < p.T;
+        tpos[i] = valid[i] ? tok % p.L : 0;       // position inside its sequence (the conv does not cross sequences)
+      }
+      __nv_bfloat16* urow = p.U + (size_t)(m0 + r0) * p.De + 8 * cg;
       int stage = 0; uint32_t phase = 0;
       for (int kc = 0; kc < nkc; ++kc) {
-        const int c0 = kc * BLOCK_K + 16 * cg;    // first channel of this thread in the layer
-        // taps and bias of these 16 channels (L1-resident), requested before the wait for the H block
-        uint4 wq[4][2];
+        const int c0 = kc * BLOCK_K + 8 * cg;     // first channel of this thread in the layer
+        // taps and bias of these 8 channels (L1-resident), requested before the wait for the H block
+        float wv[KCONV][8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          if (j < p.k) {
-            const uint4* wp = reinterpret_cast<const uint4*>(p.w_conv + (size_t)j * p.De + c0);
-            wq[j][0] = __ldg(wp); wq[j][1] = __ldg(wp + 1);
-          }
-        }
-        float acc[16];
+        for (int j = 0; j < KCONV; ++j) unpack8(__ldg(reinterpret_cast<const uint4*>(p.w_conv + (size_t)j * p.De + c0)), wv[j]);
+        float acc[2][8];
         if (p.b_conv) {
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.b_conv + c0)), b1 = __ldg(reinterpret_cast<const float4*>(p.b_conv + c0) + 1);
+          const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float4 b4 = __ldg(reinterpret_cast<const float4*>(p.b_conv + c0) + i);
-            acc[4 * i] = b4.x; acc[4 * i + 1] = b4.y; acc[4 * i + 2] = b4.z; acc[4 * i + 3] = b4.w;
-          }
+          for (int i = 0; i < 8; ++i) { acc[0][i] = bb[i]; acc[1][i] = bb[i]; }
         } else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+          for (int i = 0; i < 8; ++i) { acc[0][i] = 0.0f; acc[1][i] = 0.0f; }
         }
         // the H block of this stage has landed (the producer reused the stage only after its MMAs were done)
         if (!__all_sync(0xffffffffu, mbar_wait(fullB(stage), phase, abort_flag, wait_limit))) { ok = false; break; }
         unsigned char* sa = smem + stage * F_STAGE1;
         const unsigned char* hs = sa + FA_BYTES + FB1_BYTES;      // row i of the block = token m0 - 3 + i
+        // block rows r0 + i, i = 0..4, are tokens r0 - 3 + i: row i is tap i + KCONV - 4 of token r0 and tap i + KCONV - 5 of token r0 + 1
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int back = p.k - 1 - j;
-          if (j < p.k && valid && t - back >= 0) {
-            const int hr = r + F_HALO - back;
-            const uint4 h0 = *reinterpret_cast<const uint4*>(hs + hr * 128 + (((2 * cg) ^ (hr & 7)) << 4));
-            const uint4 h1 = *reinterpret_cast<const uint4*>(hs + hr * 128 + (((2 * cg + 1) ^ (hr & 7)) << 4));
-            float hv[8], wv[8];
-            unpack8(h0, hv); unpack8(wq[j][0], wv);
+        for (int i = 0; i < 5; ++i) {
+          constexpr int K4 = KCONV - 4, K5 = KCONV - 5;
+          if (i + K4 < 0 && i + K5 < 0) continue;
+          const int hr = r0 + i;
+          float hv[8];
+          unpack8(*reinterpret_cast<const uint4*>(hs + hr * 128 + ((cg ^ (hr & 7)) << 4)), hv);
+          if (i + K4 >= 0 && i + K4 < KCONV && valid[0] && tpos[0] - (3 - i) >= 0) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = fmaf(wv[i], hv[i], acc[i]);
-            unpack8(h1, hv); unpack8(wq[j][1], wv);
+            for (int c = 0; c < 8; ++c) acc[0][c] = fmaf(wv[(i + K4) < 0 ? 0 : (i + K4) >= KCONV ? 0 : (i + K4)][c], hv[c], acc[0][c]);
+          }
+          if (i + K5 >= 0 && i + K5 < KCONV && valid[1] && tpos[1] - (4 - i) >= 0) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[8 + i] = fmaf(wv[i], hv[i], acc[8 + i]);
+            for (int c = 0; c < 8; ++c) acc[1][c] = fmaf(wv[(i + K5) < 0 ? 0 : (i + K5) >= KCONV ? 0 : (i + K5)][c], hv[c], acc[1][c]);
           }
         }
-        float o0[8], o1[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { o0[i] = valid ? silu_fast(acc[i]) : 0.0f; o1[i] = valid ? silu_fast(acc[8 + i]) : 0.0f; }
-        const uint4 q0 = pack8(o0), q1 = pack8(o1);
-        if (valid) {
-          uint4* up = reinterpret_cast<uint4*>(urow + (size_t)kc * BLOCK_K);
-          up[0] = q0; up[1] = q1;
+        for (int i = 0; i < 2; ++i) {
+          float o[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) o[c] = valid[i] ? silu_fast(acc[i][c]) : 0.0f;
+          const uint4 q = pack8(o);
+          if (valid[i]) *reinterpret_cast<uint4*>(urow + (size_t)i * p.De + (size_t)kc * BLOCK_K) = q;
+          const int r = r0 + i;
+          *reinterpret_cast<uint4*>(sa + r * 128 + ((cg ^ (r & 7)) << 4)) = q;
         }
-        *reinterpret_cast<uint4*>(sa + sw0) = q0;
-        *reinterpret_cast<uint4*>(sa + sw1) = q1;
         fence_async_smem();                      // generic-proxy writes -> visible to the tensor core's reads
         __syncwarp();
         if (lane == 0) mbar_arrive(fullA(stage));
@@ -301,7 +303,7 @@ fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_c
       tc_fence_after();
       const int row = quarter * 32 + lane;
       const int tok = m0 + row;
-      const bool valid = tok < p.T;
+      const bool valid = row < p.rows_cta && tok < p.T;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
       for (int ch = part; ch * 32 < p.block_n1; ch += 4) {
         uint32_t ra[32];
@@ -359,7 +361,7 @@ fused_conv_xdt_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_c
         }
         if (n_pieces > 0) {
           __syncwarp();
-          softplus_flush_bf16<EPI_SOFTPLUS>(ep, stage_out, m0 + quarter * 32, p.T, n_base + c0 * 32, p.De, n_pieces, lane);
+          softplus_flush_bf16<EPI_SOFTPLUS>(ep, stage_out, m0 + quarter * 32, min(p.T, m0 + p.rows_cta), n_base + c0 * 32, p.De, n_pieces, lane);
           __syncwarp();
         }
         tc_fence_before();
@@ -402,12 +404,21 @@ cudaError_t launch_fused_conv_xdt(const rom_config& c, const void* HZ, int ldh, 
   if (!make_tmap(&twdt, W_dt, (uint64_t)De, (uint64_t)R, (uint64_t)R, (uint32_t)block_n3)) return cudaErrorInvalidValue;
   // instruction descriptors: D = f32, A = B = bf16, both K-major, N >> 3 at bit 17, M >> 4 at bit 24
   auto idesc = [](int n) { return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24); };
+  // tokens per CTA: the fewest waves of 128-token tiles, then the rows spread evenly over the SMs of those waves
+  int num_sms = 0;
+  cudaError_t e = current_device_sm_count(&num_sms);
+  if (e != cudaSuccess) return e;
+  const long long waves = ((long long)T + (long long)BLOCK_M * num_sms - 1) / ((long long)BLOCK_M * num_sms);
+  int rows_cta = (int)((T + waves * num_sms - 1) / (waves * num_sms));
+  rows_cta = (rows_cta + 7) / 8 * 8;
+  if (rows_cta > BLOCK_M) rows_cta = BLOCK_M;
   const FusedArgs a{static_cast<const __nv_bfloat16*>(HZ), ldh, static_cast<const __nv_bfloat16*>(w_conv), b_conv, b_dt,
                     static_cast<__nv_bfloat16*>(U), static_cast<__nv_bfloat16*>(delta_r), Bm, Cm, static_cast<__nv_bfloat16*>(Delta),
-                    T, c.L, De, R, N, c.d_conv, block_n1, block_n3};
-  cudaError_t e = cudaFuncSetAttribute(fused_conv_xdt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);
+                    T, c.L, De, R, N, c.d_conv, block_n1, block_n3, rows_cta};
+  auto kern = c.d_conv == 4 ? fused_conv_xdt_kernel<4> : c.d_conv == 3 ? fused_conv_xdt_kernel<3> : fused_conv_xdt_kernel<2>;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);
   if (e != cudaSuccess) return e;
-  fused_conv_xdt_kernel<<<(T + BLOCK_M - 1) / BLOCK_M, F_THREADS, F_SMEM, st>>>(th, twx, twdt, a, idesc(block_n1), idesc(block_n3), status, WAIT_LIMIT);
+  kern<<<(T + rows_cta - 1) / rows_cta, F_THREADS, F_SMEM, st>>>(th, twx, twdt, a, idesc(block_n1), idesc(block_n3), status, WAIT_LIMIT);
   count_launch();
   return cudaGetLastError();
 }
