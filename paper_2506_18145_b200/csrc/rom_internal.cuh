@@ -185,6 +185,13 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, b
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
                         void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st);
 
+// One-pass scan for few long sequences (rom_scan_seq.cu): every exponential evaluated once, no workspace.  bf16 storage only.
+bool scan_seq_applicable(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* Bm, const float* Cm,
+                         const void* z, int ldz, const int32_t* z_row, const int32_t* y_rows, int K, int num_sms);
+cudaError_t launch_scan_seq(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
+                            const float* Cm, const float* D, const void* z, int ldz, const float* h0, void* y, float* h_last,
+                            const int32_t* y_rows, int K, bool gate_activated, cudaStream_t st);
+
 // Backward of the scan (gradients of every input); ckpt: scan_bwd_ws_bytes() bytes of scratch.  dA, dBm, dCm, dD are
 // zeroed here and accumulated with atomics.  z / dz, h0, dh_last, dD, dh0 may be null.
 size_t scan_bwd_ws_bytes(int B, int De, int L);

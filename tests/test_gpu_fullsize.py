@@ -58,6 +58,8 @@ def test_layer_full_size_benchmark_inputs():
 @pytest.mark.parametrize("B,L,De,disc_mode,use_ws", [
     (1, 16384, 4096, 0, True),       # the launch bench.py --stage scan times: 10 chunks, two launches + state chain
     (1, 16384, 4096, 1, True),
+    (1, 16384, 4096, 0, False),      # no workspace: one pass at one warp per scheduler, every exponential evaluated once
+    (1, 16384, 4096, 1, False),
     (64, 1024, 3072, 0, False),      # short_seqs shape: one pass, 8 states per thread
 ])
 def test_scan_full_size(B, L, De, disc_mode, use_ws):
