@@ -6,10 +6,10 @@
 //   [z|x|B|C|dt]_t = sum_i 1_i X_t W_in,i;  (x,B,C) <- SiLU(conv(x,B,C));  dt = softplus(dt + dt_bias);
 //   per head h:  H_t = exp(dt A_h) H_{t-1} + dt x_t (x) B_t,  y_t = C_t H_t + D_h x_t;
 //   y^ = RMSNorm(y * SiLU(z)) * w_norm;  O_t = sum_i R_i y^_t W_out,i.
-// Launch sequence: the RoM layer's router / permutation / gather, the grouped GEMM, the slot sum, a conv over the
-// x|B|C slab, a per-head dt expansion, the selective-scan kernel (the scalar-per-head recurrence is its special case
+// Launch sequence: the RoM layer's router / permutation / gather, the grouped GEMM (rows back in token order at top-1 on
+// the tensor path, otherwise a sum over the slots), a conv over the x|B|C slab, a per-head dt expansion, the selective-scan kernel (the scalar-per-head recurrence is its special case
 // A[c, n] = A_head(c), Delta[t, c] = dt[t, head(c)], B-bar = Delta B), a row-wise gated RMS norm that writes the rows in
-// expert order, the grouped output GEMM and the gate-weighted combine.  A first version: parity first, not tuned.
+// expert order, the grouped output GEMM and the gate-weighted combine.
 #include "rom_internal.cuh"
 
 namespace rom {
@@ -76,31 +76,100 @@ int check_m2(const rom_config* c, int headdim) {
   return ROM_OK;
 }
 
-// SiLU(conv) over the x | B | C slab of the token-order projection rows: one thread per (token, channel).
+// 16 bytes of consecutive elements as floats
+template <typename T> struct V16;
+template <> struct V16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  uint4 q;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ __forceinline__ void zero() { q = make_uint4(0, 0, 0, 0); }
+  __device__ __forceinline__ void get(float (&v)[8]) const {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+  }
+  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8]) {
+    uint4 o;
+    uint32_t* w = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]); w[i] = *reinterpret_cast<const uint32_t*>(&h); }
+    *reinterpret_cast<uint4*>(p) = o;
+  }
+};
+template <> struct V16<float> {
+  static constexpr int N = 4;
+  float4 q;
+  __device__ __forceinline__ void load(const float* p) { q = __ldg(reinterpret_cast<const float4*>(p)); }
+  __device__ __forceinline__ void zero() { q = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+  __device__ __forceinline__ void get(float (&v)[4]) const { v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
+  static __device__ __forceinline__ void store(float* p, const float (&v)[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+};
+
+constexpr int M2_TCH = 16;      // tokens per thread of the conv kernel
+
+// SiLU(conv) over the x | B | C slab of the token-order projection rows.  A thread owns one 16-byte group of channels
+// and M2_TCH consecutive tokens of one sequence: the M2_TCH + 3 rows it needs are requested at once.
 //   ZXs [T, W]: columns [De, 2De + 2N) are the slab; x part -> xc [T, De] (dtype), B, C parts -> Bm, Cm [T, N] (fp32).
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 m2_conv_kernel(const T* __restrict__ ZXs, const T* __restrict__ w_conv, const float* __restrict__ b_conv, T* __restrict__ xc,
-               float* __restrict__ Bm, float* __restrict__ Cm, int L, int De, int N, int W, int k, long long total) {
-  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
+               float* __restrict__ Bm, float* __restrict__ Cm, int L, int De, int N, int W, int k) {
+  constexpr int V = V16<T>::N;
   const int Cs = De + 2 * N;
-  const long long tok = i / Cs;
-  const int ch = (int)(i % Cs);
-  const int t = (int)(tok % L);
-  float acc = b_conv ? b_conv[ch] : 0.0f;
-  for (int j = 0; j < k; ++j) {
-    const int back = (k - 1) - j;
-    if (t - back >= 0) acc = fmaf(to_f32(w_conv[(size_t)j * Cs + ch]), to_f32(ZXs[(tok - back) * W + De + ch]), acc);
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * V;
+  if (c0 >= Cs) return;
+  const int tb = blockIdx.y * M2_TCH;
+  const size_t tok0 = (size_t)blockIdx.z * L;
+  constexpr int NR = M2_TCH + 3;
+  V16<T> raw[NR];
+#pragma unroll
+  for (int r = 0; r < NR; ++r) {
+    const int t = tb - 3 + r;
+    if (t >= 0 && t < L) raw[r].load(ZXs + (tok0 + t) * W + De + c0);
+    else raw[r].zero();
   }
-  const float v = sizeof(T) == 4 ? acc / (1.0f + expf(-acc)) : silu_fast(acc);
-  if (ch < De) xc[tok * De + ch] = from_f32<T>(v);
-  else if (ch < De + N) Bm[tok * N + (ch - De)] = v;
-  else Cm[tok * N + (ch - De - N)] = v;
+  // taps right-aligned into 4 slots: slot 3 multiplies the current token
+  float w[4][V], bias[V];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int src = j - (4 - k);
+    if (src >= 0) { V16<T> t; t.load(w_conv + (size_t)src * Cs + c0); t.get(w[j]); }
+    else {
+#pragma unroll
+      for (int i = 0; i < V; ++i) w[j][i] = 0.0f;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < V; ++i) bias[i] = b_conv ? b_conv[c0 + i] : 0.0f;
+#pragma unroll
+  for (int r = 0; r < M2_TCH; ++r) {
+    const int t = tb + r;
+    if (t >= L) break;
+    float acc[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = bias[i];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float hv[V];
+      raw[r + j].get(hv);
+#pragma unroll
+      for (int i = 0; i < V; ++i) acc[i] = fmaf(w[j][i], hv[i], acc[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) acc[i] = sizeof(T) == 4 ? acc[i] / (1.0f + expf(-acc[i])) : silu_fast(acc[i]);
+    const size_t tok = tok0 + t;
+    if (c0 < De) {
+      V16<T>::store(xc + tok * De + c0, acc);
+    } else {
+      float* dst = c0 < De + N ? Bm + tok * N + (c0 - De) : Cm + tok * N + (c0 - De - N);
+#pragma unroll
+      for (int i = 0; i < V; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+    }
+  }
 }
 
-// Delta[t, c] = softplus(dt_raw[t, head(c)] + dt_bias[head(c)]) expanded over the head's channels (fp32);
-// block 0 also expands A_h, D_h to the per-(channel, state) / per-channel arrays the scan kernel reads.
+// Delta[t, c] = softplus(dt_raw[t, head(c)] + dt_bias[head(c)]) expanded over the head's channels (fp32), four channels
+// per thread; the first threads also expand A_h, D_h to the per-(channel, state) / per-channel arrays the scan kernel reads.
 template <typename T>
 __global__ void __launch_bounds__(256)
 m2_dt_kernel(const T* __restrict__ ZXs, const float* __restrict__ dt_bias, const float* __restrict__ A, const float* __restrict__ D,
@@ -111,23 +180,31 @@ m2_dt_kernel(const T* __restrict__ ZXs, const float* __restrict__ dt_bias, const
     for (int n = 0; n < N; ++n) A_exp[i * N + n] = A[h];
     D_exp[i] = D ? D[h] : 0.0f;
   }
-  if (i >= Tn * De) return;
-  const long long tok = i / De;
-  const int c = (int)(i % De), h = c / headdim;
-  const float v = to_f32(ZXs[tok * W + 2 * De + 2 * N + h]) + (dt_bias ? dt_bias[h] : 0.0f);
-  D32[i] = softplus_f(v);
+  const int q4 = De / 4;
+  if (i >= Tn * q4) return;
+  const long long tok = i / q4;
+  const int c = (int)(i % q4) * 4, h = c / headdim;       // headdim is a multiple of 8: the four channels share a head
+  const float v = softplus_f(to_f32(ZXs[tok * W + 2 * De + 2 * N + h]) + (dt_bias ? dt_bias[h] : 0.0f));
+  *reinterpret_cast<float4*>(D32 + tok * De + c) = make_float4(v, v, v, v);
 }
 
-// y^ = g / sqrt(mean g^2 + eps) * w_norm with g = the gated scan output of the token (one block per token), written to the
-// K expert-order rows of the token.
+// y^ = g / sqrt(mean g^2 + eps) * w_norm with g = the gated scan output of the token (one block per token, 16-byte
+// accesses), written to the K expert-order rows of the token.
 template <typename T>
 __global__ void __launch_bounds__(256)
 m2_norm_kernel(const T* __restrict__ Yt, const float* __restrict__ w_norm, const int32_t* __restrict__ row_of_assign, T* __restrict__ Ygp,
                int De, int K, float eps) {
+  constexpr int V = V16<T>::N;
   __shared__ float red[8];
   const size_t t = blockIdx.x;
+  const int nvec = De / V;
   float ss = 0.0f;
-  for (int c = threadIdx.x; c < De; c += blockDim.x) { const float v = to_f32(Yt[t * De + c]); ss = fmaf(v, v, ss); }
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    V16<T> q; q.load(Yt + t * De + (size_t)i * V);
+    float v[V]; q.get(v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) ss = fmaf(v[j], v[j], ss);
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -136,9 +213,12 @@ m2_norm_kernel(const T* __restrict__ Yt, const float* __restrict__ w_norm, const
 #pragma unroll
   for (int i = 0; i < 8; ++i) tot += red[i];
   const float r = rsqrtf(tot / (float)De + eps);
-  for (int c = threadIdx.x; c < De; c += blockDim.x) {
-    const T v = from_f32<T>(to_f32(Yt[t * De + c]) * r * w_norm[c]);
-    for (int k = 0; k < K; ++k) Ygp[(size_t)row_of_assign[t * K + k] * De + c] = v;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    V16<T> q; q.load(Yt + t * De + (size_t)i * V);
+    float v[V]; q.get(v);
+#pragma unroll
+    for (int j = 0; j < V; ++j) v[j] = to_f32(from_f32<T>(v[j] * r * w_norm[(size_t)i * V + j]));
+    for (int k = 0; k < K; ++k) V16<T>::store(Ygp + (size_t)row_of_assign[t * K + k] * De + (size_t)i * V, v);
   }
 }
 
@@ -200,22 +280,29 @@ int rom_mamba2_layer_forward(const rom_config* cfg, int32_t headdim, const rom_m
   ROM_CUDA(cudaMemsetAsync(status, 0, sizeof(int32_t) * kStatusInts, st));
   ROM_CUDA(launch_route_gather(c, x, w->W_r, w->b_r, topk_idx_out, gates, counts_out, W, lay, st));
   // fused input projection of the selected experts, then the sum over a token's slots (indicator only)
-  Epilogue e_in{EPI_STORE, W + m.ZXp, Wd, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
-  ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_in, Dm, (int64_t)Wd * Dm, Wd, Dm, e_in));
-  ROM_CUDA(launch_slot_sum(c.dtype, W + m.ZXp, row_of_assign, W + m.ZXs, T, Wd, c.K, st));
+  if (tc && c.K == 1) {
+    // one expert per token: the output op writes every row straight to its token's position (no activation: R = width)
+    Epilogue e_in{EPI_INPROJ, W + m.ZXs, Wd, nullptr, nullptr, nullptr, Wd, 0, reinterpret_cast<const int32_t*>(W + lay.assign_of_row), nullptr};
+    ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_in, Dm, (int64_t)Wd * Dm, Wd, Dm, e_in));
+  } else {
+    Epilogue e_in{EPI_STORE, W + m.ZXp, Wd, nullptr, nullptr, nullptr, 0, 0, nullptr, nullptr};
+    ROM_CUDA(gemm(W + lay.x_perm, Dm, w->W_in, Dm, (int64_t)Wd * Dm, Wd, Dm, e_in));
+    ROM_CUDA(launch_slot_sum(c.dtype, W + m.ZXp, row_of_assign, W + m.ZXs, T, Wd, c.K, st));
+  }
   // shared conv + SiLU over x | B | C; dt per head
   {
-    const long long total = (long long)T * (De + 2 * N);
-    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const int Cs = De + 2 * N;
+    const int vec = bf ? 8 : 4;
+    dim3 cgrid((Cs / vec + 127) / 128, (c.L + M2_TCH - 1) / M2_TCH, c.B);
     float* Bm = reinterpret_cast<float*>(W + m.Bm);
     float* Cm = reinterpret_cast<float*>(W + m.Cm);
-    if (bf) m2_conv_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)(W + m.ZXs), (const __nv_bfloat16*)w->w_conv, w->b_conv,
-                                                                 (__nv_bfloat16*)(W + m.xc), Bm, Cm, c.L, De, N, Wd, c.d_conv, total);
-    else m2_conv_kernel<float><<<blocks, 256, 0, st>>>((const float*)(W + m.ZXs), (const float*)w->w_conv, w->b_conv, (float*)(W + m.xc), Bm, Cm,
-                                                     c.L, De, N, Wd, c.d_conv, total);
+    if (bf) m2_conv_kernel<__nv_bfloat16><<<cgrid, 128, 0, st>>>((const __nv_bfloat16*)(W + m.ZXs), (const __nv_bfloat16*)w->w_conv, w->b_conv,
+                                                                (__nv_bfloat16*)(W + m.xc), Bm, Cm, c.L, De, N, Wd, c.d_conv);
+    else m2_conv_kernel<float><<<cgrid, 128, 0, st>>>((const float*)(W + m.ZXs), (const float*)w->w_conv, w->b_conv, (float*)(W + m.xc), Bm, Cm,
+                                                    c.L, De, N, Wd, c.d_conv);
     count_launch();
     ROM_CUDA(cudaGetLastError());
-    const long long total2 = (long long)T * De;
+    const long long total2 = max((long long)T * (De / 4), (long long)De);
     const unsigned blocks2 = (unsigned)((total2 + 255) / 256);
     float* D32 = reinterpret_cast<float*>(W + m.D32);
     float* A_exp = reinterpret_cast<float*>(W + m.A_exp);
