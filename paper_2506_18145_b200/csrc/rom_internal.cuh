@@ -183,7 +183,8 @@ cudaError_t launch_conv_step(const rom_config& c, const void* XZp, const int32_t
 // delta: [B, L, d_inner], fp32 when delta_fp32, else in the storage dtype.
 cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
-                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st);
+                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st,
+                        bool scalar_A = false /* A[c, :] constant per channel and disc_mode 1: one exponential per channel and step */);
 
 // One-pass scan for few long sequences (rom_scan_seq.cu): every exponential evaluated once, no workspace.  bf16 storage only.
 bool scan_seq_applicable(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* Bm, const float* Cm,

@@ -316,7 +316,7 @@ int rom_mamba2_layer_forward(const rom_config* cfg, int32_t headdim, const rom_m
     rom_config cs = c;
     cs.disc_mode = 1;
     ROM_CUDA(launch_scan(cs, W + m.xc, D32, true, A_exp, Bm, Cm, w->D ? D_exp : nullptr, W + m.ZXs, Wd, nullptr, nullptr, W + m.Yt, nullptr,
-                         nullptr, 1, reinterpret_cast<float*>(W + m.scan_ws), false, st));
+                         nullptr, 1, reinterpret_cast<float*>(W + m.scan_ws), false, st, true));
   }
   // gated RMS norm, rows written in expert order
   if (bf) m2_norm_kernel<__nv_bfloat16><<<T, 256, 0, st>>>((const __nv_bfloat16*)(W + m.Yt), w->w_norm, row_of_assign, (__nv_bfloat16*)(W + m.Ygp), De, c.K, 1e-5f);

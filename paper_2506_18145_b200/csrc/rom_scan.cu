@@ -121,6 +121,8 @@ struct ScanArgs {
   float* sum_delta;     // state-only blocks: [B*nch, De] sum of Delta over the chunk
   int gate_activated;   // z already holds SiLU(gate pre-activation): multiply only
   int chunk_off;        // chunk of blockIdx.z == 0
+  int scalar_a;         // A[c, :] is one value per channel (scalar-per-head decay of a Mamba2-style block): one exponential
+                        // per channel and step instead of one per state (only with B-bar = Delta B)
 };
 // TD: type Delta is stored in: float (the rom_scan entry point, the fp32 layer) or the storage type (bf16 layer).
 
@@ -277,8 +279,9 @@ scan_kernel(const ScanArgs p) {
     float* __restrict__ psp = ps;
     constexpr int UF = S > 4 ? S : (NC * NS >= 16 ? 2 : 4);
     float held = 0.0f;      // the even step's partial sum, kept for the paired exchange (S == 2)
-    auto tile_steps = [&](auto so_tag) {
+    auto tile_steps = [&](auto so_tag, auto sc_tag) {
     constexpr bool STATE_ONLY = decltype(so_tag)::value;
+    constexpr bool SCALAR_A = decltype(sc_tag)::value && !ZOH;
 #pragma unroll UF
     for (int tt = 0; tt < TS; ++tt) {
       float4 bc[NP];
@@ -291,10 +294,18 @@ scan_kernel(const ScanArgs p) {
         const float2 dl2 = make_float2(dv.x, dv.y), vv2 = make_float2(dv.z, dv.w);
         if (STATE_ONLY) sdel[i] += dv.x;
         float2 acc0 = make_float2(0.0f, 0.0f), acc1 = make_float2(0.0f, 0.0f);
+        float a_all = 0.0f;
+        if (SCALAR_A) a_all = PRECISE ? expf(dl2.x * a2[i][0].x) : ex2_approx(dl2.x * a2[i][0].x);
 #pragma unroll
         for (int q = 0; q < NP; ++q) {
           const float2 Bv = make_float2(bc[q].x, bc[q].y), Cv = make_float2(bc[q].z, bc[q].w);
-          if (PRECISE) {
+          if (SCALAR_A) {
+            h[i][q] = __ffma2_rn(make_float2(a_all, a_all), h[i][q], __fmul2_rn(vv2, Bv));      // w = (Delta u) B
+            if (!STATE_ONLY) {
+              float2& acc = (q & 1) ? acc1 : acc0;
+              acc = q < 2 ? __fmul2_rn(Cv, h[i][q]) : __ffma2_rn(Cv, h[i][q], acc);
+            }
+          } else if (PRECISE) {
             const float dA0 = dl2.x * a2[i][q].x, dA1 = dl2.x * a2[i][q].y;
             // B-bar u: zero-order hold expm1(dA)/A * B * u, or (Delta u) * B
             const float w0 = ZOH ? -expm1f(dA0) * kin[i][q].x * Bv.x * vv2.x : Bv.x * vv2.x;
@@ -322,7 +333,7 @@ scan_kernel(const ScanArgs p) {
             }
           }
         }
-        if (NP > 1 && !PRECISE) acc0 = __fadd2_rn(acc0, acc1);
+        if (NP > 1 && (!PRECISE || SCALAR_A)) acc0 = __fadd2_rn(acc0, acc1);
         part[i] = acc0.x + acc0.y;
       }
       if (STATE_ONLY) {
@@ -369,10 +380,13 @@ scan_kernel(const ScanArgs p) {
     }
 
     };
-    if (MODE == 0) tile_steps(std::false_type{});
-    else if (MODE == 1) tile_steps(std::true_type{});
-    else if (so) tile_steps(std::true_type{});
-    else tile_steps(std::false_type{});
+    if (p.scalar_a) {
+      if (MODE == 1 || (MODE == 2 && so)) tile_steps(std::true_type{}, std::true_type{});
+      else tile_steps(std::false_type{}, std::true_type{});
+    } else {
+      if (MODE == 1 || (MODE == 2 && so)) tile_steps(std::true_type{}, std::false_type{});
+      else tile_steps(std::false_type{}, std::false_type{});
+    }
 
     if (more) stash(tiles[buf ^ 1]);
     __syncthreads();
@@ -562,16 +576,17 @@ cudaError_t launch_scan_t(const rom_config& c, ScanArgs a, const float* A, const
 
 cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                         const float* Cm, const float* D, const void* z, int ldz, const int32_t* z_row, const float* h0,
-                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st) {
+                        void* y, float* h_last, const int32_t* y_rows, int K, float* chunk_ws, bool gate_activated, cudaStream_t st,
+                        bool scalar_A) {
   int num_sms = 0;
   const cudaError_t e = current_device_sm_count(&num_sms);
   if (e != cudaSuccess) return e;
   // Few long sequences and no workspace for the chunked scan: the one-pass low-occupancy kernel (every exponential once;
   // 0.69 ms against 1.04 ms for one 16384-step sequence of 4096 channels).  With a workspace the two chunked launches
   // below are as fast (0.70 ms), so they stay the path of the layer.
-  if (chunk_ws == nullptr && scan_seq_applicable(c, u, delta, delta_fp32, Bm, Cm, z, ldz, z_row, y_rows, K, num_sms))
+  if (chunk_ws == nullptr && !scalar_A && scan_seq_applicable(c, u, delta, delta_fp32, Bm, Cm, z, ldz, z_row, y_rows, K, num_sms))
     return launch_scan_seq(c, u, delta, delta_fp32, A, Bm, Cm, D, z, ldz, h0, y, h_last, y_rows, K, gate_activated, st);
-  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0};
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0, (scalar_A && c.disc_mode == 1) ? 1 : 0};
   if (c.dtype != ROM_BF16) return launch_scan_t<float, float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
   return delta_fp32 ? launch_scan_t<__nv_bfloat16, float, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
                     : launch_scan_t<__nv_bfloat16, __nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
