@@ -193,6 +193,10 @@ cudaError_t launch_scan_seq(const rom_config& c, const void* u, const void* delt
                             const float* Cm, const float* D, const void* z, int ldz, const float* h0, void* y, float* h_last,
                             const int32_t* y_rows, int K, bool gate_activated, cudaStream_t st);
 
+// State recurrence alone over uniform chunks (rom_scan.cu; used by the backward pass): see the definition.
+cudaError_t launch_scan_states(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm, int Lc, int ncc,
+                               const float* h_in, float* h_end, float* sum_delta, float* ckpt, int nck, cudaStream_t st);
+
 // Backward of the scan (gradients of every input); ckpt: scan_bwd_ws_bytes() bytes of scratch.  dA, dBm, dCm, dD are
 // zeroed here and accumulated with atomics.  z / dz, h0, dh_last, dD, dh0 may be null.
 size_t scan_bwd_ws_bytes(int B, int De, int L);

@@ -121,6 +121,8 @@ struct ScanArgs {
   float* sum_delta;     // state-only blocks: [B*nch, De] sum of Delta over the chunk
   int gate_activated;   // z already holds SiLU(gate pre-activation): multiply only
   int chunk_off;        // chunk of blockIdx.z == 0
+  float* ckpt;          // MODE 3: [B, nck, De, 16] state at the start of every 16 steps (nck per sequence)
+  int nck;
   int scalar_a;         // A[c, :] is one value per channel (scalar-per-head decay of a Mamba2-style block): one exponential
                         // per channel and step instead of one per state (only with B-bar = Delta B)
 };
@@ -129,7 +131,8 @@ struct ScanArgs {
 // PRECISE: libm-accurate exp / expm1 (fp32 configuration, 1e-4 tolerance); otherwise one ex2.approx per
 // state update (bf16 configurations, 2e-2 tolerance).
 // ZOH: zero-order-hold B-bar (disc_mode 0); otherwise B-bar = Delta B.
-// MODE 0: full scan.  MODE 1: state only (no outputs, only h_last and sum_delta of every chunk).  MODE 2: first
+// MODE 0: full scan.  MODE 1: state only (no outputs, only h_last and sum_delta of every chunk).  MODE 3: state only
+// from the given chunk-start states, storing the state at the start of every 16 steps (backward pass).  MODE 2: first
 // launch of the chunked scan: chunk 0 runs the full scan from the caller's initial state (h0 indexed by
 // sequence), the other chunks run state-only from a zero state.
 template <typename T, typename TD, int NC, int NS, bool PRECISE, bool ZOH, int MODE>
@@ -149,7 +152,7 @@ scan_kernel(const ScanArgs p) {
   const int De = p.De, K = p.K;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int chunk = blockIdx.z + p.chunk_off;
-  const bool so = MODE == 1 || (MODE == 2 && chunk != 0);  // this block only produces its end state
+  const bool so = MODE == 1 || MODE == 3 || (MODE == 2 && chunk != 0);  // this block only produces states
   const T* __restrict__ z = so ? nullptr : static_cast<const T*>(p.z);
   const int t_first = chunk == 0 ? 0 : p.L0 + (chunk - 1) * p.Lc;
   const int L = min(chunk == 0 ? p.L0 : p.Lc, p.L - t_first);   // steps of this chunk (<= 0: an empty chunk)
@@ -267,6 +270,16 @@ scan_kernel(const ScanArgs p) {
   for (int t0 = 0; t0 < L; t0 += TS, buf ^= 1) {
     const bool more = t0 + TS < L;
     if (more) fetch(t0 + TS);
+    if constexpr (MODE == 3) {
+      static_assert(MODE != 3 || (TS == 16 && NC == 1), "one checkpoint per tile");
+      const int c = c_base + cl;
+      if (c < De) {
+        float* dst = p.ckpt + (((size_t)blockIdx.y * p.nck + (size_t)((t_first + t0) >> 4)) * De + c) * NST + g * NS;
+#pragma unroll
+        for (int q = 0; q < NP; q += 2)
+          *reinterpret_cast<float4*>(dst + 2 * q) = make_float4(h[0][q].x, h[0][q].y, h[0][q + 1].x, h[0][q + 1].y);
+      }
+    }
     const TileT& tl = tiles[buf];
     float* ys = ysum + buf * TS * YP;
 
@@ -380,11 +393,13 @@ scan_kernel(const ScanArgs p) {
     }
 
     };
-    if (p.scalar_a) {
-      if (MODE == 1 || (MODE == 2 && so)) tile_steps(std::true_type{}, std::true_type{});
+    if (MODE == 1 || MODE == 3) {
+      tile_steps(std::true_type{}, std::false_type{});
+    } else if (p.scalar_a) {
+      if (MODE == 2 && so) tile_steps(std::true_type{}, std::true_type{});
       else tile_steps(std::false_type{}, std::true_type{});
     } else {
-      if (MODE == 1 || (MODE == 2 && so)) tile_steps(std::true_type{}, std::false_type{});
+      if (MODE == 2 && so) tile_steps(std::true_type{}, std::false_type{});
       else tile_steps(std::false_type{}, std::false_type{});
     }
 
@@ -407,7 +422,7 @@ scan_kernel(const ScanArgs p) {
         p.h_last[((size_t)b * De + c) * NST + n] = h[i][q].x;
         p.h_last[((size_t)b * De + c) * NST + n + 1] = h[i][q].y;
       }
-      if (so && g == 0) p.sum_delta[(size_t)b * De + c] = sdel[i];
+      if (so && g == 0 && p.sum_delta) p.sum_delta[(size_t)b * De + c] = sdel[i];
     }
   }
 }
@@ -586,10 +601,29 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, b
   // below are as fast (0.70 ms), so they stay the path of the layer.
   if (chunk_ws == nullptr && !scalar_A && scan_seq_applicable(c, u, delta, delta_fp32, Bm, Cm, z, ldz, z_row, y_rows, K, num_sms))
     return launch_scan_seq(c, u, delta, delta_fp32, A, Bm, Cm, D, z, ldz, h0, y, h_last, y_rows, K, gate_activated, st);
-  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0, (scalar_A && c.disc_mode == 1) ? 1 : 0};
+  const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0, nullptr, 0, (scalar_A && c.disc_mode == 1) ? 1 : 0};
   if (c.dtype != ROM_BF16) return launch_scan_t<float, float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
   return delta_fp32 ? launch_scan_t<__nv_bfloat16, float, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st)
                     : launch_scan_t<__nv_bfloat16, __nv_bfloat16, false>(c, a, A, h0, h_last, chunk_ws, num_sms, st);
+}
+
+// State recurrence alone over uniform chunks of Lc steps (Lc a multiple of 16; ncc chunks per sequence), for the backward pass.
+// ckpt == nullptr: every chunk from a zero state; h_end [B, ncc, De, 16] and sum_delta [B, ncc, De] leave.
+// ckpt != nullptr: every chunk from its true start state h_in [B, ncc, De, 16] (null: zero); the state at the start of every
+// 16 steps is stored to ckpt [B, nck, De, 16].
+cudaError_t launch_scan_states(const rom_config& c, const void* u, const float* delta, const float* A, const float* Bm, int Lc, int ncc,
+                               const float* h_in, float* h_end, float* sum_delta, float* ckpt, int nck, cudaStream_t st) {
+  ScanArgs a{u, delta, A, Bm, /* C is fetched with B but not used */ Bm, nullptr, nullptr, 0, nullptr, h_in, nullptr, h_end, nullptr, 1, c.L, c.d_inner, Lc, ncc, Lc, sum_delta,
+             0, 0, ckpt, nck, 0};
+  const bool zoh = c.disc_mode == 0;
+  if (ckpt == nullptr) {
+    a.h0 = nullptr;
+    if (c.dtype != ROM_BF16) return zoh ? launch_one<float, float, 1, 8, true, true, 1>(a, c.B, ncc, st) : launch_one<float, float, 1, 8, true, false, 1>(a, c.B, ncc, st);
+    return zoh ? launch_one<__nv_bfloat16, float, 1, 8, false, true, 1>(a, c.B, ncc, st) : launch_one<__nv_bfloat16, float, 1, 8, false, false, 1>(a, c.B, ncc, st);
+  }
+  a.h_last = nullptr;
+  if (c.dtype != ROM_BF16) return zoh ? launch_one<float, float, 1, 8, true, true, 3>(a, c.B, ncc, st) : launch_one<float, float, 1, 8, true, false, 3>(a, c.B, ncc, st);
+  return zoh ? launch_one<__nv_bfloat16, float, 1, 8, false, true, 3>(a, c.B, ncc, st) : launch_one<__nv_bfloat16, float, 1, 8, false, false, 3>(a, c.B, ncc, st);
 }
 
 }  // namespace rom

@@ -5,8 +5,8 @@
 // Reverse, with g = dLoss/dh_t carried from later steps and e_t = dout_t * SiLU(z_t):
 //           g += C_t e_t;  dC_t = sum_c e_t h_t;  dA-bar = g h_{t-1};  db = g u_t;  du_t = sum_n g b + D e_t;  g <- a_t g.
 //
-// The reverse sweep needs h_{t-1} and h_t at every step.  A first kernel runs the recurrence forward and keeps the
-// state at the start of every chunk of 16 steps (checkpoints in the workspace).  The second kernel walks the chunks
+// The reverse sweep needs h_{t-1} and h_t at every step.  First the forward scan kernel runs the recurrence in its
+// state-only mode and keeps the state at the start of every chunk of 16 steps (checkpoints in the workspace).  The second kernel walks the chunks
 // backwards: it recomputes the chunk's states from its checkpoint into shared memory, then sweeps the chunk in
 // reverse.  A thread owns 4 of the 16 states of one channel of one sequence (4 adjacent lanes per channel): sums over
 // the states (dDelta, du, the forward y for the gate's derivative) are shuffles over those lanes; sums over channels
@@ -54,55 +54,6 @@ __device__ __forceinline__ void exp_and_expm1(float x, float& ex, float& em1) {
 }
 template <bool PRECISE>
 __device__ __forceinline__ float exp_only(float x) { return PRECISE ? expf(x) : ex2_ftz(1.4426950408889634f * x); }
-
-// Forward pass that only records the state at the start of every chunk.
-template <typename T, bool ZOH>
-__global__ void __launch_bounds__(BT)
-scan_ckpt_kernel(const BwdArgs p) {
-  const int tid = threadIdx.x, cl = tid >> 2, q = tid & 3;
-  const int c = blockIdx.x * BCH + cl;
-  const size_t b = blockIdx.y;
-  if (c >= p.De) return;
-  const T* __restrict__ u = static_cast<const T*>(p.u);
-  const int cj = blockIdx.z;
-  const int t_lo = cj * p.Lc, t_hi = min(t_lo + p.Lc, p.L);
-  float a[4], h[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    a[i] = p.A[(size_t)c * NST + 4 * q + i];
-    if (p.ncc > 1) h[i] = p.h_in[((b * p.ncc + cj) * p.De + c) * NST + 4 * q + i];
-    else h[i] = p.h0 ? p.h0[(b * p.De + c) * NST + 4 * q + i] : 0.0f;
-  }
-  constexpr bool PRECISE = sizeof(T) == 4;
-  float ia[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) ia[i] = 1.0f / a[i];
-  for (int t4 = t_lo; t4 < t_hi; t4 += 4) {       // CK is a multiple of 4: a checkpoint falls on the first step of a group
-    float dl[4], uu[4];
-    float4 B4[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {                 // the group's loads first
-      const int t = min(t4 + j, t_hi - 1);
-      const size_t e = (b * p.L + t) * p.De + c;
-      dl[j] = p.delta[e]; uu[j] = to_f32(u[e]);
-      B4[j] = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
-    }
-    if ((t4 % CK) == 0)
-      *reinterpret_cast<float4*>(p.ckpt + ((b * p.nck + t4 / CK) * p.De + c) * NST + 4 * q) = make_float4(h[0], h[1], h[2], h[3]);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (t4 + j >= t_hi) break;
-      const float bv[4] = {B4[j].x, B4[j].y, B4[j].z, B4[j].w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float ex, em1;
-        exp_and_expm1<PRECISE>(dl[j] * a[i], ex, em1);
-        const float bb = ZOH ? em1 * ia[i] * bv[i] : dl[j] * bv[i];
-        h[i] = fmaf(ex, h[i], bb * uu[j]);
-      }
-    }
-  }
-}
 
 template <typename T, bool ZOH>
 __global__ void __launch_bounds__(BT)
@@ -300,9 +251,10 @@ scan_bwd_kernel(const BwdArgs p) {
 }
 
 
-// Pre-pass of the chunk-parallel form, one coarse chunk per blockIdx.z: from a zero state the chunk's end state and sum
-// of Delta; from a zero gradient the gradient that leaves the chunk's start (g <- a_t (g + C_t e_t), t descending).
-template <typename T, bool ZOH>
+// Pre-pass of the chunk-parallel form, one coarse chunk per blockIdx.z: from a zero gradient, the gradient that leaves the
+// chunk's start (g <- a_t (g + C_t e_t), t descending).  (The chunk's end state and sum of Delta from a zero state come
+// from the forward scan kernel's state-only mode.)
+template <typename T>
 __global__ void __launch_bounds__(BT)
 scan_bwd_prepass_kernel(const BwdArgs p) {
   const int tid = threadIdx.x, cl = tid >> 2, q = tid & 3;
@@ -311,65 +263,36 @@ scan_bwd_prepass_kernel(const BwdArgs p) {
   if (c >= p.De) return;
   const int cj = blockIdx.z;
   const int t_lo = cj * p.Lc, t_hi = min(t_lo + p.Lc, p.L);
-  const T* __restrict__ u = static_cast<const T*>(p.u);
   const T* __restrict__ dy = static_cast<const T*>(p.dy);
   const T* __restrict__ z = static_cast<const T*>(p.z);
-  float a[4], h[4] = {0.0f, 0.0f, 0.0f, 0.0f}, g[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  float a[4], g[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
   for (int i = 0; i < 4; ++i) a[i] = p.A[(size_t)c * NST + 4 * q + i];
   constexpr bool PRECISE = sizeof(T) == 4;
-  float ia[4];
+  constexpr int G = 8;                            // steps whose loads are in flight together
+  for (int t4 = t_hi - 1; t4 >= t_lo; t4 -= G) {
+    float dl[G], ev[G], zz[G];
+    float4 C4[G];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) ia[i] = 1.0f / a[i];
-  float sd = 0.0f;
-  for (int t4 = t_lo; t4 < t_hi; t4 += 4) {
-    float dl[4], uu[4];
-    float4 B4[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int t = min(t4 + j, t_hi - 1);
-      const size_t e = (b * p.L + t) * p.De + c;
-      dl[j] = p.delta[e]; uu[j] = to_f32(u[e]);
-      B4[j] = *reinterpret_cast<const float4*>(p.Bm + (b * p.L + t) * NST + 4 * q);
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if (t4 + j >= t_hi) break;
-      const float bv[4] = {B4[j].x, B4[j].y, B4[j].z, B4[j].w};
-      sd += dl[j];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float ex, em1;
-        exp_and_expm1<PRECISE>(dl[j] * a[i], ex, em1);
-        const float bb = ZOH ? em1 * ia[i] * bv[i] : dl[j] * bv[i];
-        h[i] = fmaf(ex, h[i], bb * uu[j]);
-      }
-    }
-  }
-  for (int t4 = t_hi - 1; t4 >= t_lo; t4 -= 4) {
-    float dl[4], ev[4];
-    float4 C4[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < G; ++j) {
       const int t = max(t4 - j, t_lo);
       const size_t e = (b * p.L + t) * p.De + c;
       dl[j] = p.delta[e];
       ev[j] = to_f32(dy[e]);
-      if (z) { const float zz = to_f32(z[(b * p.L + t) * p.ldz + c]); ev[j] *= zz * sigmoid_f(zz); }
+      zz[j] = z ? to_f32(z[(b * p.L + t) * p.ldz + c]) : 0.0f;
       C4[j] = *reinterpret_cast<const float4*>(p.Cm + (b * p.L + t) * NST + 4 * q);
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < G; ++j) {
       if (t4 - j < t_lo) break;
+      if (z) ev[j] *= zz[j] * sigmoid_f(zz[j]);
       const float cv[4] = {C4[j].x, C4[j].y, C4[j].z, C4[j].w};
 #pragma unroll
       for (int i = 0; i < 4; ++i) g[i] = fmaf(cv[i], ev[j], g[i]) * exp_only<PRECISE>(dl[j] * a[i]);
     }
   }
   const size_t o = ((b * p.ncc + cj) * p.De + c) * NST + 4 * q;
-  *reinterpret_cast<float4*>(p.h_end + o) = make_float4(h[0], h[1], h[2], h[3]);
   *reinterpret_cast<float4*>(p.q_start + o) = make_float4(g[0], g[1], g[2], g[3]);
-  if (q == 0) p.sum_delta[(b * p.ncc + cj) * p.De + c] = sd;
 }
 
 // Composes the coarse chunks (both recurrences are linear): with P_j = exp(A sum_delta_j),
@@ -450,11 +373,9 @@ cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void
   const dim3 grid((c.d_inner + BCH - 1) / BCH, c.B, ncc);
   const bool zoh = c.disc_mode == 0, bf = c.dtype == ROM_BF16;
   if (ncc > 1) {
-    if (bf) {
-      if (zoh) scan_bwd_prepass_kernel<__nv_bfloat16, true><<<grid, BT, 0, st>>>(a); else scan_bwd_prepass_kernel<__nv_bfloat16, false><<<grid, BT, 0, st>>>(a);
-    } else {
-      if (zoh) scan_bwd_prepass_kernel<float, true><<<grid, BT, 0, st>>>(a); else scan_bwd_prepass_kernel<float, false><<<grid, BT, 0, st>>>(a);
-    }
+    // chunk end states and sums of Delta from a zero state (forward scan kernel, state-only), chunk-start gradients from zero
+    if ((e = launch_scan_states(c, u, delta, A, Bm, Lc, ncc, nullptr, h_end, sum_delta, nullptr, 0, st)) != cudaSuccess) return e;
+    if (bf) scan_bwd_prepass_kernel<__nv_bfloat16><<<grid, BT, 0, st>>>(a); else scan_bwd_prepass_kernel<float><<<grid, BT, 0, st>>>(a);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     const long long n_thr = (long long)c.B * c.d_inner * NST;
@@ -462,13 +383,8 @@ cudaError_t launch_scan_backward(const rom_config& c, const void* dy, const void
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  if (bf) {
-    if (zoh) scan_ckpt_kernel<__nv_bfloat16, true><<<grid, BT, 0, st>>>(a); else scan_ckpt_kernel<__nv_bfloat16, false><<<grid, BT, 0, st>>>(a);
-  } else {
-    if (zoh) scan_ckpt_kernel<float, true><<<grid, BT, 0, st>>>(a); else scan_ckpt_kernel<float, false><<<grid, BT, 0, st>>>(a);
-  }
-  count_launch();
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  // the state at the start of every 16 steps, from the true chunk-start states (forward scan kernel, state-only)
+  if ((e = launch_scan_states(c, u, delta, A, Bm, Lc, ncc, ncc > 1 ? h_in : h0, nullptr, nullptr, ckpt, nck, st)) != cudaSuccess) return e;
   auto kern = bf ? (zoh ? scan_bwd_kernel<__nv_bfloat16, true> : scan_bwd_kernel<__nv_bfloat16, false>)
                  : (zoh ? scan_bwd_kernel<float, true> : scan_bwd_kernel<float, false>);
   if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BWD_SMEM)) != cudaSuccess) return e;
