@@ -108,15 +108,33 @@ combine_bwd_kernel(const T* __restrict__ dYgu, const T* __restrict__ Ygp, const 
   int rows[kMaxK]; float g[kMaxK], part[kMaxK];
   for (int k = 0; k < K; ++k) { rows[k] = row_of_assign[t * K + k]; g[k] = gates[t * K + k]; part[k] = 0.0f; }
   const T* yg = Ygp + (size_t)rows[0] * De;          // the K rows of a token hold the same gated scan output
-  for (int c = threadIdx.x; c < De; c += blockDim.x) {
-    const float y = to_f32(yg[c]);
-    float acc = 0.0f;
-    for (int k = 0; k < K; ++k) {
-      const float b = to_f32(dYgu[(size_t)rows[k] * De + c]);
-      acc = fmaf(g[k], b, acc);
-      part[k] = fmaf(b, y, part[k]);
+  constexpr int V = V16<T>::N;
+  if (De % V == 0) {                                   // 16-byte accesses
+    for (int i = threadIdx.x; i < De / V; i += blockDim.x) {
+      V16<T> q;
+      float y[V], acc[V];
+      q.load(yg + (size_t)i * V); q.get(y);
+#pragma unroll
+      for (int j = 0; j < V; ++j) acc[j] = 0.0f;
+      for (int k = 0; k < K; ++k) {
+        float bv[V];
+        q.load(dYgu + (size_t)rows[k] * De + (size_t)i * V); q.get(bv);
+#pragma unroll
+        for (int j = 0; j < V; ++j) { acc[j] = fmaf(g[k], bv[j], acc[j]); part[k] = fmaf(bv[j], y[j], part[k]); }
+      }
+      V16<T>::store(dYg + t * De + (size_t)i * V, acc);
     }
-    dYg[t * De + c] = from_f32<T>(acc);
+  } else {
+    for (int c = threadIdx.x; c < De; c += blockDim.x) {
+      const float y = to_f32(yg[c]);
+      float acc = 0.0f;
+      for (int k = 0; k < K; ++k) {
+        const float b = to_f32(dYgu[(size_t)rows[k] * De + c]);
+        acc = fmaf(g[k], b, acc);
+        part[k] = fmaf(b, y, part[k]);
+      }
+      dYg[t * De + c] = from_f32<T>(acc);
+    }
   }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int k = 0; k < K; ++k) {
@@ -183,23 +201,37 @@ conv_bwd_kernel(const T* __restrict__ HZ, const T* __restrict__ w_conv, const fl
     const int t = t0 - k + j;
     hw[j] = t >= 0 ? to_f32(HZ[(tok0 + t) * ld + c]) : 0.0f;
   }
-  for (int t = t0; t < t_end; ++t) {
-    for (int j = 0; j + 1 < k; ++j) hw[j] = hw[j + 1];
-    hw[k - 1] = to_f32(HZ[(tok0 + t) * ld + c]);
-    float pre = bias;
-    for (int j = 0; j < k; ++j) pre = fmaf(w[j], hw[j], pre);
-    const float sg = 1.0f / (1.0f + expf(-pre));
-    const float g = (to_f32(dU1[(tok0 + t) * De + c]) + to_f32(dU2[(tok0 + t) * De + c])) * sg * (1.0f + pre * (1.0f - sg));
-    if (t < t1) {
-      dbl += g;
-      for (int j = 0; j < k; ++j) dwl[j] = fmaf(g, hw[j], dwl[j]);
+  constexpr int G = 8;                      // steps whose loads are in flight together
+  for (int tg = t0; tg < t_end; tg += G) {
+    float hz[G], d1[G], d2[G];
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+      const int t = min(tg + i, t_end - 1);
+      hz[i] = to_f32(HZ[(tok0 + t) * ld + c]);
+      d1[i] = to_f32(dU1[(tok0 + t) * De + c]);
+      d2[i] = to_f32(dU2[(tok0 + t) * De + c]);
     }
-    // dacc[i] collects dH of step t - (k-1) + i; after this step's terms, index 0 is complete
-    for (int j = 0; j < k; ++j) dacc[j] = fmaf(w[j], g, dacc[j]);
-    const int tau = t - (k - 1);
-    if (tau >= t0) dHZ[(tok0 + tau) * ld + c] = from_f32<T>(dacc[0]);
-    for (int j = 0; j + 1 < k; ++j) dacc[j] = dacc[j + 1];
-    dacc[k - 1] = 0.0f;
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+      const int t = tg + i;
+      if (t >= t_end) break;
+      for (int j = 0; j + 1 < k; ++j) hw[j] = hw[j + 1];
+      hw[k - 1] = hz[i];
+      float pre = bias;
+      for (int j = 0; j < k; ++j) pre = fmaf(w[j], hw[j], pre);
+      const float sg = 1.0f / (1.0f + expf(-pre));
+      const float g = (d1[i] + d2[i]) * sg * (1.0f + pre * (1.0f - sg));
+      if (t < t1) {
+        dbl += g;
+        for (int j = 0; j < k; ++j) dwl[j] = fmaf(g, hw[j], dwl[j]);
+      }
+      // dacc[i] collects dH of step t - (k-1) + i; after this step's terms, index 0 is complete
+      for (int j = 0; j < k; ++j) dacc[j] = fmaf(w[j], g, dacc[j]);
+      const int tau = t - (k - 1);
+      if (tau >= t0) dHZ[(tok0 + tau) * ld + c] = from_f32<T>(dacc[0]);
+      for (int j = 0; j + 1 < k; ++j) dacc[j] = dacc[j + 1];
+      dacc[k - 1] = 0.0f;
+    }
   }
   // steps whose later neighbours do not exist (end of the sequence): what has been collected is final
   for (int i = 0; i + 1 < k; ++i) {

@@ -76,35 +76,6 @@ int check_m2(const rom_config* c, int headdim) {
   return ROM_OK;
 }
 
-// 16 bytes of consecutive elements as floats
-template <typename T> struct V16;
-template <> struct V16<__nv_bfloat16> {
-  static constexpr int N = 8;
-  uint4 q;
-  __device__ __forceinline__ void load(const __nv_bfloat16* p) { q = __ldg(reinterpret_cast<const uint4*>(p)); }
-  __device__ __forceinline__ void zero() { q = make_uint4(0, 0, 0, 0); }
-  __device__ __forceinline__ void get(float (&v)[8]) const {
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-  }
-  static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&v)[8]) {
-    uint4 o;
-    uint32_t* w = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]); w[i] = *reinterpret_cast<const uint32_t*>(&h); }
-    *reinterpret_cast<uint4*>(p) = o;
-  }
-};
-template <> struct V16<float> {
-  static constexpr int N = 4;
-  float4 q;
-  __device__ __forceinline__ void load(const float* p) { q = __ldg(reinterpret_cast<const float4*>(p)); }
-  __device__ __forceinline__ void zero() { q = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
-  __device__ __forceinline__ void get(float (&v)[4]) const { v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w; }
-  static __device__ __forceinline__ void store(float* p, const float (&v)[4]) { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
-};
-
 constexpr int M2_TCH = 16;      // tokens per thread of the conv kernel
 
 // SiLU(conv) over the x | B | C slab of the token-order projection rows.  A thread owns one 16-byte group of channels
