@@ -188,7 +188,7 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, b
 
 // One-pass scan for few long sequences (rom_scan_seq.cu): every exponential evaluated once, no workspace.  bf16 storage only.
 bool scan_seq_applicable(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* Bm, const float* Cm,
-                         const void* z, int ldz, const int32_t* z_row, const int32_t* y_rows, int K, int num_sms);
+                         const void* z, int ldz, const int32_t* z_row, const int32_t* y_rows, bool gate_activated, int num_sms);
 cudaError_t launch_scan_seq(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* A, const float* Bm,
                             const float* Cm, const float* D, const void* z, int ldz, const float* h0, void* y, float* h_last,
                             const int32_t* y_rows, int K, bool gate_activated, cudaStream_t st);

@@ -24,9 +24,11 @@
 // converts and stores it to the other shared buffer.  The scan proper leaves sum_n C h in shared
 // memory; the skip term, the gate, the rounding and the 16-byte row stores are done by the thread
 // that loaded that piece, which still holds u and z in registers.  One __syncthreads per tile.  The
-// per-channel operands are stored duplicated, (Delta, Delta, v, v), so one 16-byte load yields both
-// packed operands; 8-channel groups are XOR-swizzled so that loader stores and compute loads are
-// both bank-conflict free.
+// per-channel operands are stored once, (Delta, v), and duplicated into packed pairs in registers: the
+// path that returns shared-memory data to the register file (128 bytes per clock per SM, one copy per
+// lane whatever the sharing) is as busy as the special-function unit in this kernel, so every byte
+// counts; the channel pairs of an 8-channel group are rotated so that loader stores and compute loads
+// are both bank-conflict free.
 #include <type_traits>
 
 #include <cmath>
@@ -103,12 +105,14 @@ struct Geo {
 };
 
 // position of channel c inside its tile row: the 8 channels of a group are permuted by the group index
-__device__ __forceinline__ int swz(int c) { return (c & ~7) | ((c ^ (c >> 3)) & 7); }
+// (the four channel pairs of a group are rotated by half the group index: a loader thread's four 16-byte stores then
+// fall into different banks than its neighbours')
+__device__ __forceinline__ int swz(int c) { return (c & ~7) | ((((c >> 1) + (c >> 4)) & 3) << 1) | (c & 1); }
 
 // Shared-memory image of one input tile.
 template <int NC, int NS>
 struct Tile {
-  float4 dv[Geo<NC, NS>::TS][Geo<NC, NS>::CH];   // (Delta, Delta, v, v) at [t][swz(c)]: v = u (zero-order hold) or Delta*u
+  float2 dv[Geo<NC, NS>::TS][Geo<NC, NS>::CH];   // (Delta, v) at [t][swz(c)]: v = u (zero-order hold) or Delta*u
   float4 bc[Geo<NC, NS>::TS][NST / 2];           // (B_n, B_n+1, C_n, C_n+1) per state pair
 };
 
@@ -222,11 +226,11 @@ scan_kernel(const ScanArgs p) {
   auto stash = [&](TileT& tl) {     // registers -> shared, converting
     float d[8], uu[8];
     pre_d.get(d); pre_u.get(uu);
-    float4* row = &tl.dv[lr][lc];
+    float4* row = reinterpret_cast<float4*>(&tl.dv[lr][lc]);       // the group's four channel pairs
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const float v = ZOH ? uu[i] : d[i] * uu[i];
-      row[i ^ ((lc >> 3) & 7)] = make_float4(d[i], d[i], v, v);
+    for (int i = 0; i < 4; ++i) {
+      const float v0 = ZOH ? uu[2 * i] : d[2 * i] * uu[2 * i], v1 = ZOH ? uu[2 * i + 1] : d[2 * i + 1] * uu[2 * i + 1];
+      row[(i + (lc >> 4)) & 3] = make_float4(d[2 * i], v0, d[2 * i + 1], v1);
     }
 #pragma unroll
     for (int i = 0; i < G::NBC; ++i) reinterpret_cast<float*>(&tl.bc[warp + 8 * i][0])[bc_dst] = pre_bc[i];
@@ -286,7 +290,7 @@ scan_kernel(const ScanArgs p) {
     // Plain loop over the steps of the tile: loads, exponentials and the recurrence of one step in
     // program order, unrolled a few steps so the scheduler can overlap them.  The restrict-qualified
     // views tell the compiler that the stores of the sums never alias the tile it reads.
-    const float4* __restrict__ dvp = &tl.dv[0][0];
+    const float2* __restrict__ dvp = &tl.dv[0][0];
     const float4* __restrict__ bcp = &tl.bc[0][g * NP];
     float* __restrict__ ysp = ys + cl;
     float* __restrict__ psp = ps;
@@ -303,8 +307,8 @@ scan_kernel(const ScanArgs p) {
       float part[NC];
 #pragma unroll
       for (int i = 0; i < NC; ++i) {
-        const float4 dv = dvp[tt * CH + cl_sw[i]];
-        const float2 dl2 = make_float2(dv.x, dv.y), vv2 = make_float2(dv.z, dv.w);
+        const float2 dv = dvp[tt * CH + cl_sw[i]];
+        const float2 dl2 = make_float2(dv.x, dv.x), vv2 = make_float2(dv.y, dv.y);
         if (STATE_ONLY) sdel[i] += dv.x;
         float2 acc0 = make_float2(0.0f, 0.0f), acc1 = make_float2(0.0f, 0.0f);
         float a_all = 0.0f;
@@ -599,7 +603,7 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, b
   // Few long sequences and no workspace for the chunked scan: the one-pass low-occupancy kernel (every exponential once;
   // 0.69 ms against 1.04 ms for one 16384-step sequence of 4096 channels).  With a workspace the two chunked launches
   // below are as fast (0.70 ms), so they stay the path of the layer.
-  if (chunk_ws == nullptr && !scalar_A && scan_seq_applicable(c, u, delta, delta_fp32, Bm, Cm, z, ldz, z_row, y_rows, K, num_sms))
+  if (chunk_ws == nullptr && !scalar_A && scan_seq_applicable(c, u, delta, delta_fp32, Bm, Cm, z, ldz, z_row, y_rows, gate_activated, num_sms))
     return launch_scan_seq(c, u, delta, delta_fp32, A, Bm, Cm, D, z, ldz, h0, y, h_last, y_rows, K, gate_activated, st);
   const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0, nullptr, 0, (scalar_A && c.disc_mode == 1) ? 1 : 0};
   if (c.dtype != ROM_BF16) return launch_scan_t<float, float, true>(c, a, A, h0, h_last, chunk_ws, num_sms, st);

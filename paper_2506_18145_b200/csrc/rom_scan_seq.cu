@@ -307,16 +307,8 @@ cudaError_t launch_seq_k(const SeqArgs& a, int B, cudaStream_t st) {
 }
 template <typename TD, bool ZOH>
 cudaError_t launch_seq_t(const SeqArgs& a, int B, cudaStream_t st) {
-  const int gate = a.z == nullptr ? 0 : (a.gate_activated ? 1 : 2);
-  const bool rows = a.y_rows != nullptr;
-  switch (gate * 2 + (rows ? 1 : 0)) {
-    case 0: return launch_seq_k<TD, ZOH, 0, false>(a, B, st);
-    case 1: return launch_seq_k<TD, ZOH, 0, true>(a, B, st);
-    case 2: return launch_seq_k<TD, ZOH, 1, false>(a, B, st);
-    case 3: return launch_seq_k<TD, ZOH, 1, true>(a, B, st);
-    case 4: return launch_seq_k<TD, ZOH, 2, false>(a, B, st);
-    default: return launch_seq_k<TD, ZOH, 2, true>(a, B, st);
-  }
+  // the entry point that reaches this kernel passes the raw gate (or none) and writes rows in token order
+  return a.z == nullptr ? launch_seq_k<TD, ZOH, 0, false>(a, B, st) : launch_seq_k<TD, ZOH, 2, false>(a, B, st);
 }
 
 bool aligned16p(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -324,8 +316,8 @@ bool aligned16p(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) =
 }  // namespace
 
 bool scan_seq_applicable(const rom_config& c, const void* u, const void* delta, bool delta_fp32, const float* Bm, const float* Cm,
-                         const void* z, int ldz, const int32_t* z_row, const int32_t* y_rows, int K, int num_sms) {
-  if (y_rows != nullptr && K != 1) return false;
+                         const void* z, int ldz, const int32_t* z_row, const int32_t* y_rows, bool gate_activated, int num_sms) {
+  if (y_rows != nullptr || (z != nullptr && gate_activated)) return false;      // only the plain forms are instantiated
   if (c.dtype != ROM_BF16 || c.d_state != NST || c.L < 2 || z_row != nullptr) return false;
   if (c.d_inner % Q_CH != 0 || (z && ldz % Q_CH != 0)) return false;
   if (!aligned16p(u) || !aligned16p(delta) || !aligned16p(Bm) || !aligned16p(Cm) || (z && !aligned16p(z))) return false;
