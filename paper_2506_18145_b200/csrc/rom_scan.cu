@@ -296,6 +296,7 @@ scan_kernel(const ScanArgs p) {
     float* __restrict__ psp = ps;
     constexpr int UF = S > 4 ? S : (NC * NS >= 16 ? 2 : 4);
     float held = 0.0f;      // the even step's partial sum, kept for the paired exchange (S == 2)
+    float pend_keep = 0.0f, pend_recv = 0.0f;   // the exchange of the previous pair, finished one pair later (S == 2)
     auto tile_steps = [&](auto so_tag, auto sc_tag) {
     constexpr bool STATE_ONLY = decltype(so_tag)::value;
     constexpr bool SCALAR_A = decltype(sc_tag)::value && !ZOH;
@@ -364,8 +365,10 @@ scan_kernel(const ScanArgs p) {
         if ((tt & 1) == 0) {
           held = part[0];
         } else {
-          const float recv = __shfl_xor_sync(0xffffffffu, g ? held : part[0], 1);
-          ysp[(tt - 1 + g) * YP] = (g ? part[0] : held) + recv;
+          // the sum of the previous pair is stored only now: its shuffle has had two steps to complete
+          if (tt > 1) ysp[(tt - 3 + g) * YP] = pend_keep + pend_recv;
+          pend_recv = __shfl_xor_sync(0xffffffffu, g ? held : part[0], 1);
+          pend_keep = g ? part[0] : held;
         }
       } else if (S <= 4) {
         // all S lanes of the channel get the sum; lane g stores the steps with tt % S == g
@@ -407,6 +410,7 @@ scan_kernel(const ScanArgs p) {
       else tile_steps(std::false_type{}, std::false_type{});
     }
 
+    if (S == 2 && NC == 1 && !so) ysp[(TS - 2 + g) * YP] = pend_keep + pend_recv;      // the tile's last pair
     if (more) stash(tiles[buf ^ 1]);
     __syncthreads();
     if (!so) {
