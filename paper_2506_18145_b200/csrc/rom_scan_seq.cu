@@ -134,7 +134,7 @@ scan_seq_kernel(const SeqArgs p) {
   // runs stage 1 of group k+2, stage 2 of group k+1, ... stage 6 of group k-3: every producer of a long-latency result
   // (shared-memory load, exponential, shuffle) is a whole iteration ahead of its consumer.
   //   S1 raw operand loads;  S2 conversions, exponentials, input terms w;  S3 the recurrence and the partial sums C h;
-  //   S4, S5 the two rounds of the exchange that finishes the sums;  S6 skip term, gate, rounding, store.
+  //   S4, S5 the two steps of the exchange that finishes the sums;  S6 skip term, gate, rounding, store.
   struct Raw {
     TD d[4];
     __nv_bfloat16 u[4];
@@ -147,8 +147,8 @@ scan_seq_kernel(const SeqArgs p) {
     float4 C4[4];
   };
   struct Meta { float ue, ze; int row; };
-  struct X1 { float k0, k1, r0, r1; Meta m; };       // kept partial sums and what the partner sent (round 1)
-  struct X2 { float k, r; Meta m; };                 // the same for round 2
+  struct X1 { float k0, k1, r0, r1; Meta m; };       // kept partial sums and what the partner sent (first exchange)
+  struct X2 { float k, r; Meta m; };                 // the same for the second exchange
 
   auto S1 = [&](int grp, Raw& o) {
     const Stage& s = stages[(grp >> 3) % Q_STAGES];
