@@ -169,8 +169,10 @@ ROM_API int rom_route_noalloc(const rom_config *cfg, const void *x, const void *
  *   u, z, y : [B, L, d_inner] dtype;  delta : [B, L, d_inner] fp32;  A : [d_inner, d_state] fp32;
  *   Bm, Cm : [B, L, d_state] fp32;  D : [d_inner] or NULL;  z NULL = no gate;
  *   h0 : [B, d_inner, d_state] fp32 or NULL (zeros);  h_last : same shape or NULL (not produced).
- *   ws : NULL (one pass per sequence, whatever its length) or at least rom_scan_workspace_size(cfg) bytes
- *        (a larger buffer, e.g. the layer's workspace, is accepted; only its head is used).
+ *   ws : NULL (one pass per sequence, whatever its length; with few long bf16 sequences a kernel built for one warp per
+ *        SM sub-partition is used) or at least rom_scan_workspace_size(cfg) bytes (few long sequences are then cut into
+ *        chunks scanned in parallel; a larger buffer, e.g. the layer's workspace, is accepted; only its head is used).
+ *        The result does not depend on the choice beyond fp32 rounding order.
  * Uses cfg->B, L, d_inner, d_state, dtype, disc_mode.                                             */
 ROM_API int rom_scan(const rom_config *cfg, const void *u, const float *delta, const float *A,
              const float *Bm, const float *Cm, const float *D, const void *z, const float *h0,
