@@ -279,6 +279,20 @@ def run_stage(args, s):
     for _ in range(max(args.warmup, 3)):
         call()
     torch.cuda.synchronize()
+    if args.graph:
+        # the entry points allocate nothing and never synchronise, so a call can be captured once and replayed
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            call()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            call()
+        direct, call = call, graph.replay
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
@@ -289,6 +303,8 @@ def run_stage(args, s):
     line = {"stage": args.stage, "workload": s.name, "ms": ms, "algorithmic_bytes": nbytes,
             "achieved_gbs": nbytes / ms / 1e6, "hbm_peak_gbs": peaks["hbm_gbs"], "frac": nbytes / ms / 1e6 / peaks["hbm_gbs"],
             "peak_source": peaks["source"]}
+    if args.graph:
+        line["cuda_graph"] = True
     if "step_batch" in extra:
         line["sequences"] = extra["step_batch"]
         line["tokens_per_s"] = extra["step_batch"] / ms * 1e3
@@ -323,6 +339,7 @@ def main():
     ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
                     help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
                          "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
+    ap.add_argument("--graph", action="store_true", help="with --stage: capture one call in a CUDA graph and time its replay")
     ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn", "step", "backward", "mamba2"],
                     help="layer: the whole forward (the benchmark); scan / route / ffn / step: that entry point alone, timed in isolation "
                          "at the workload's shape (kernel studies and ncu captures; prints a short JSON line)")
