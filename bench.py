@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 # Each entry names the source files of its kernel and the SHA-256 prefix of their contents at capture time: when a file
 # has changed since, the counters are stale and are reported as null.
 NCU_CAPTURES = {
-    ("scan", "long_ctx"): {"traffic": 748.2e6, "sources": ["rom_scan.cu"], "sha": "1c10fcc4ac14"},
+    ("scan", "long_ctx"): {"traffic": 748.2e6, "sources": ["rom_scan.cu"], "sha": "27a64847762c"},
     ("in_proj", "long_ctx"): {"traffic": 601.1e6, "tensor_pipe_active_pct": 72.8, "sources": ["rom_gemm_tc.cu", "rom_tc_ptx.cuh"], "sha": "12dc3b87707f"},
 }
 NOMINAL_PEAKS = {"hbm_gbs": 7700.0, "bf16_tflops": 2250.0}      # datasheet figures, for context beside the measured ones
@@ -196,7 +196,8 @@ def run_stage(args, s):
         q = synth.make_scan_inputs(s.B, s.L, s.d_inner, s.d_state, s.dtype, s.seed_base + 500)
         d = {k: (None if v is None else v.to(dev)) for k, v in q.items()}
         y = torch.empty_like(d["u"])
-        ws = torch.empty(max(rb.scan_workspace_size(cfg), 16), dtype=torch.uint8, device=dev)
+        # with a workspace a long sequence is scanned as parallel chunks; without one (--no-scan-ws) in one pass
+        ws = None if args.no_scan_ws else torch.empty(max(rb.scan_workspace_size(cfg), 16), dtype=torch.uint8, device=dev)
         call = lambda: rb.rom_scan(cfg, d["u"], d["delta"], d["A"], d["Bm"], d["Cm"], d["D"], d["z"], None, y, None, ws)
         esz = 2 if s.dtype == "bf16" else 4
         nbytes = s.T * (4 * s.d_inner * esz + 8 * s.d_state)        # u, Delta, z, y at storage width; B, C fp32
@@ -339,6 +340,7 @@ def main():
     ap.add_argument("--small-proj", default="shared", choices=["shared", "routed"],
                     help="shared: one x Proj / dt Proj for all experts (the method as proposed, the benchmark); routed: one "
                          "per expert under the same routing (the ablation row of Section 5.3; a secondary number)")
+    ap.add_argument("--no-scan-ws", action="store_true", help="with --stage scan: call rom_scan without a workspace (one pass per sequence)")
     ap.add_argument("--graph", action="store_true", help="with --stage: capture one call in a CUDA graph and time its replay")
     ap.add_argument("--stage", default="layer", choices=["layer", "scan", "route", "ffn", "step", "backward", "mamba2"],
                     help="layer: the whole forward (the benchmark); scan / route / ffn / step: that entry point alone, timed in isolation "

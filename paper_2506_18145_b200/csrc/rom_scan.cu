@@ -605,8 +605,8 @@ cudaError_t launch_scan(const rom_config& c, const void* u, const void* delta, b
   const cudaError_t e = current_device_sm_count(&num_sms);
   if (e != cudaSuccess) return e;
   // Few long sequences and no workspace for the chunked scan: the one-pass low-occupancy kernel (every exponential once;
-  // 0.69 ms against 1.04 ms for one 16384-step sequence of 4096 channels).  With a workspace the two chunked launches
-  // below are as fast (0.70 ms), so they stay the path of the layer.
+  // 0.74 ms against 1.04 ms for one 16384-step sequence of 4096 channels).  With a workspace the two chunked launches
+  // below are faster (0.67 ms), so they stay the path of the layer.
   if (chunk_ws == nullptr && !scalar_A && scan_seq_applicable(c, u, delta, delta_fp32, Bm, Cm, z, ldz, z_row, y_rows, gate_activated, num_sms))
     return launch_scan_seq(c, u, delta, delta_fp32, A, Bm, Cm, D, z, ldz, h0, y, h_last, y_rows, K, gate_activated, st);
   const ScanArgs a{u, delta, A, Bm, Cm, D, z, ldz, z_row, h0, y, h_last, y_rows, K, c.L, c.d_inner, c.L, 1, c.L, nullptr, gate_activated ? 1 : 0, 0, nullptr, 0, (scalar_A && c.disc_mode == 1) ? 1 : 0};

@@ -16,8 +16,8 @@
 //   * the sum over states of C h is finished four steps at a time by a transposing exchange (3 shuffles): lane g
 //     ends up with the sum of step g of the group, adds D u, applies the gate, rounds and stores that one value;
 //   * the loop is software-pipelined by hand over groups of four steps (six stages, see the kernel).
-// Measured on one 16384-step sequence of 4096 channels: 0.69 ms (the general kernel without a workspace: 1.04 ms; with a
-// workspace, chunked: 0.70 ms).  What binds is not the special-function unit: with every shared-memory load,
+// Measured on one 16384-step sequence of 4096 channels (fp32 Delta, raw gate): 0.74 ms (the general kernel without a
+// workspace: 1.04 ms; with a workspace, chunked: 0.67 ms).  What binds is not the special-function unit: with every shared-memory load,
 // exponential and shuffle taken out the remaining fp32 / integer stream alone needs 0.48 ms, and two sequences take
 // 1.8 x the time of one, i.e. the fp32 pipes are the limit (a packed fp32 operation occupies them for two cycles:
 // 128 lanes per clock per SM, packed or not, as measured).
@@ -263,26 +263,26 @@ scan_seq_kernel(const SeqArgs p) {
       for (int gg = 0; gg < 8; ++gg) {
         const int k = 8 * i + gg;
         X2 x2n; X1 x1n;
-        S2(rc, opn, mn);
         S6(k - 3, x2, std::true_type{});
         S5(x1, x2n);
         S4(part, mprev, x1n);
-        S1(k + 2, rn);
         S3(ops, part, std::true_type{}, 4);
         mprev = mc;
+        S2(rc, opn, mn);
+        S1(k + 2, rn);
         rc = rn; ops = opn; mc = mn; x1 = x1n; x2 = x2n;
       }
     } else {
       const int kend = min(8 * i + 8, niter);
       for (int k = 8 * i; k < kend; ++k) {
         X2 x2n; X1 x1n;
-        S2(rc, opn, mn);
         S6(k - 3, x2, std::false_type{});
         S5(x1, x2n);
         S4(part, mprev, x1n);
-        S1(k + 2, rn);
         S3(ops, part, std::false_type{}, k < nfull ? 4 : max(0, L - 4 * k));
         mprev = mc;
+        S2(rc, opn, mn);
+        S1(k + 2, rn);
         rc = rn; ops = opn; mc = mn; x1 = x1n; x2 = x2n;
       }
     }
